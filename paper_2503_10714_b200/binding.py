@@ -1,0 +1,251 @@
+"""ctypes binding of libzsm.so: the same entry points as include/zsm.h.
+
+Argument marshalling only -- every step of the path runs in the library's CUDA
+kernels.  There is no fallback: if the shared library is missing the import of
+this module raises.  torch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libzsm.so")
+
+ZSM_OK = 0
+ZSM_ERR_INVALID_ARG = 1
+ZSM_ERR_BUFFER_TOO_SMALL = 2
+ZSM_ERR_STATE = 3
+ZSM_ERR_CUDA = 4
+ZSM_ERR_UNSUPPORTED = 5
+ZSM_ERR_DEVICE_CHECK = 6
+ZSM_ERR_TIMEOUT = 7
+ZSM_F32, ZSM_F16, ZSM_BF16 = 0, 1, 2
+DTYPE_CODE = {"f32": ZSM_F32, "f16": ZSM_F16, "bf16": ZSM_BF16,
+              torch.float32: ZSM_F32, torch.float16: ZSM_F16, torch.bfloat16: ZSM_BF16}
+
+# every symbol include/zsm.h declares
+SYMBOLS = ["zsm_split_budget", "zsm_cache_bytes", "zsm_cache_create", "zsm_cache_reset",
+           "zsm_cache_free", "zsm_prefill_workspace_bytes", "zsm_prefill_compress",
+           "zsm_decode_step", "zsm_decode_staging_bytes", "zsm_decode_step_host",
+           "zsm_unit_capacity", "zsm_cache_export_unit", "zsm_cache_import_unit",
+           "zsm_last_device_status", "zsm_decode_launch_info", "zsm_status_string"]
+
+
+class ZsmConfig(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("n_q_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("dtype", C.c_int32),
+                ("budget_p", C.POINTER(C.c_int32)), ("budget_c", C.POINTER(C.c_int32)),
+                ("budget_r", C.POINTER(C.c_int32)), ("lam", C.c_float), ("alpha", C.c_float),
+                ("softmax_scale", C.c_float), ("tune_stages", C.c_int32),
+                ("tune_ctas_per_sm", C.c_int32), ("tune_consumer_warps", C.c_int32)]
+
+
+class ZsmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {zsm_status_string(status)} (status {status})")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_10714_b200.build`"
+                      " (there is no CPU or PyTorch fallback)")
+_lib = C.CDLL(LIB_PATH)
+_vp, _i32, _sz = C.c_void_p, C.c_int32, C.c_size_t
+_pi32 = C.POINTER(C.c_int32)
+_lib.zsm_status_string.restype = C.c_char_p
+_lib.zsm_status_string.argtypes = [C.c_int]
+_lib.zsm_split_budget.argtypes = [_i32, C.c_float, C.c_float, _pi32, _pi32, _pi32]
+_lib.zsm_cache_bytes.argtypes = [C.POINTER(ZsmConfig), C.POINTER(_sz)]
+_lib.zsm_cache_create.argtypes = [C.POINTER(ZsmConfig), _vp, _sz, C.POINTER(_vp)]
+_lib.zsm_cache_reset.argtypes = [_vp, _vp]
+_lib.zsm_cache_free.argtypes = [_vp]
+_lib.zsm_prefill_workspace_bytes.argtypes = [_vp, _i32, _i32, C.POINTER(_sz)]
+_lib.zsm_prefill_compress.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp,
+                                      _vp, _vp, _vp]
+_lib.zsm_decode_step.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.zsm_decode_staging_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
+_lib.zsm_decode_step_host.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.zsm_unit_capacity.argtypes = [_vp, _i32, _i32, _pi32, _pi32]
+_lib.zsm_cache_export_unit.argtypes = [_vp, _i32, _i32, _i32] + [_vp] * 8 + [_vp]
+_lib.zsm_cache_import_unit.argtypes = [_vp, _i32, _i32, _i32] + [_vp] * 8 + [_vp]
+_lib.zsm_last_device_status.argtypes = [_vp, _vp]
+_lib.zsm_decode_launch_info.argtypes = [_vp, _i32, _pi32, _pi32, _pi32]
+for _name in SYMBOLS:
+    if _name != "zsm_status_string":
+        getattr(_lib, _name).restype = C.c_int
+
+
+def _check(status: int, where: str):
+    if status != ZSM_OK:
+        raise ZsmError(status, where)
+
+
+def _stream(stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _dev(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return C.c_void_p(t.data_ptr())
+
+
+def _host(a):
+    if a is None:
+        return None
+    if isinstance(a, torch.Tensor):
+        assert not a.is_cuda and a.is_contiguous()
+        return C.c_void_p(a.data_ptr())
+    assert a.flags["C_CONTIGUOUS"]
+    return C.c_void_p(a.ctypes.data)
+
+
+def zsm_status_string(status: int) -> str:
+    return _lib.zsm_status_string(int(status)).decode()
+
+
+def zsm_split_budget(B: int, tail_ratio: float = 0.5, dense_ratio: float = 0.02):
+    bp, bc, br = C.c_int32(), C.c_int32(), C.c_int32()
+    _check(_lib.zsm_split_budget(int(B), float(tail_ratio), float(dense_ratio), C.byref(bp),
+                                 C.byref(bc), C.byref(br)), "zsm_split_budget")
+    return bp.value, bc.value, br.value
+
+
+def make_config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, dtype, budget_p, budget_c,
+                budget_r, lam=0.98, alpha=1.0, softmax_scale=0.0, tune_stages=0,
+                tune_ctas_per_sm=0, tune_consumer_warps=0):
+    """Builds a zsm_config_t; the budget arrays are kept alive on the returned object."""
+    arrs = [np.ascontiguousarray(np.asarray(a, dtype=np.int32).reshape(-1))
+            for a in (budget_p, budget_c, budget_r)]
+    cfg = ZsmConfig(int(n_layers), int(batch), int(n_q_heads), int(n_kv_heads), int(head_dim),
+                    int(DTYPE_CODE[dtype]), arrs[0].ctypes.data_as(_pi32),
+                    arrs[1].ctypes.data_as(_pi32), arrs[2].ctypes.data_as(_pi32), float(lam),
+                    float(alpha), float(softmax_scale), int(tune_stages), int(tune_ctas_per_sm),
+                    int(tune_consumer_warps))
+    cfg._keep = arrs
+    return cfg
+
+
+def zsm_cache_bytes(cfg: ZsmConfig) -> int:
+    n = _sz()
+    _check(_lib.zsm_cache_bytes(C.byref(cfg), C.byref(n)), "zsm_cache_bytes")
+    return n.value
+
+
+def zsm_cache_create(cfg: ZsmConfig, dev_buf: torch.Tensor):
+    h = _vp()
+    _check(_lib.zsm_cache_create(C.byref(cfg), _dev(dev_buf), dev_buf.numel() * dev_buf.element_size(),
+                                 C.byref(h)), "zsm_cache_create")
+    return h
+
+
+def zsm_cache_reset(cache, stream=None):
+    _check(_lib.zsm_cache_reset(cache, _stream(stream)), "zsm_cache_reset")
+
+
+def zsm_cache_free(cache):
+    _check(_lib.zsm_cache_free(cache), "zsm_cache_free")
+
+
+def zsm_prefill_workspace_bytes(cache, T: int, W: int) -> int:
+    n = _sz()
+    _check(_lib.zsm_prefill_workspace_bytes(cache, int(T), int(W), C.byref(n)),
+           "zsm_prefill_workspace_bytes")
+    return n.value
+
+
+def zsm_prefill_compress(cache, layer, K, V, Qw, scores, T, W, workspace, dbg_scores=None,
+                         dbg_evicted=None, dbg_targets=None, stream=None):
+    _check(_lib.zsm_prefill_compress(cache, int(layer), _dev(K), _dev(V), _dev(Qw), _dev(scores),
+                                     int(T), int(W), _dev(workspace),
+                                     workspace.numel() * workspace.element_size(),
+                                     _dev(dbg_scores), _dev(dbg_evicted), _dev(dbg_targets),
+                                     _stream(stream)), "zsm_prefill_compress")
+
+
+def zsm_decode_step(cache, layer, q, k_new, v_new, out, victim_pos=None, merge_slot=None,
+                    stream=None):
+    _check(_lib.zsm_decode_step(cache, int(layer), _dev(q), _dev(k_new), _dev(v_new), _dev(out),
+                                _dev(victim_pos), _dev(merge_slot), _stream(stream)),
+           "zsm_decode_step")
+
+
+def zsm_decode_staging_bytes(cache, layer) -> int:
+    n = _sz()
+    _check(_lib.zsm_decode_staging_bytes(cache, int(layer), C.byref(n)), "zsm_decode_staging_bytes")
+    return n.value
+
+
+def zsm_decode_step_host(cache, layer, q_host, k_new_host, v_new_host, out_host, staging,
+                         stream=None):
+    _check(_lib.zsm_decode_step_host(cache, int(layer), _host(q_host), _host(k_new_host),
+                                     _host(v_new_host), _host(out_host), _dev(staging),
+                                     staging.numel() * staging.element_size(), _stream(stream)),
+           "zsm_decode_step_host")
+
+
+def zsm_unit_capacity(cache, layer, h):
+    a, b = C.c_int32(), C.c_int32()
+    _check(_lib.zsm_unit_capacity(cache, int(layer), int(h), C.byref(a), C.byref(b)),
+           "zsm_unit_capacity")
+    return a.value, b.value
+
+
+def zsm_cache_export_unit(cache, layer, b, h, head_dim, stream=None):
+    """Returns a dict of numpy arrays: K, V, score, pos (live rows only), Kr, Vr, w (used
+    slots only), n_live, n_res, T."""
+    cap, br = zsm_unit_capacity(cache, layer, h)
+    K = np.empty((cap, head_dim), np.float32)
+    V = np.empty((cap, head_dim), np.float32)
+    score = np.empty(cap, np.float32)
+    pos = np.empty(cap, np.int32)
+    Kr = np.empty((br, head_dim), np.float32)
+    Vr = np.empty((br, head_dim), np.float32)
+    w = np.empty(br, np.uint32)
+    cnt = np.zeros(3, np.int32)
+    _check(_lib.zsm_cache_export_unit(cache, int(layer), int(b), int(h), _host(K), _host(V),
+                                      _host(score), _host(pos), _host(Kr), _host(Vr), _host(w),
+                                      _host(cnt), _stream(stream)), "zsm_cache_export_unit")
+    n, r = int(cnt[0]), int(cnt[1])
+    return dict(K=K[:n], V=V[:n], score=score[:n], pos=pos[:n], Kr=Kr[:r], Vr=Vr[:r], w=w[:r],
+                n_live=n, n_res=r, T=int(cnt[2]))
+
+
+def zsm_cache_import_unit(cache, layer, b, h, head_dim, state, stream=None):
+    cap, br = zsm_unit_capacity(cache, layer, h)
+    n, r = int(state["n_live"]), int(state["n_res"])
+
+    def padded(a, rows, dtype, cols=None):
+        shape = (rows,) if cols is None else (rows, cols)
+        out = np.zeros(shape, dtype)
+        out[: len(a)] = a
+        return out
+    K = padded(state["K"], cap, np.float32, head_dim)
+    V = padded(state["V"], cap, np.float32, head_dim)
+    score = padded(state["score"], cap, np.float32)
+    pos = padded(state["pos"], cap, np.int32)
+    Kr = padded(state["Kr"], br, np.float32, head_dim)
+    Vr = padded(state["Vr"], br, np.float32, head_dim)
+    w = padded(state["w"], br, np.uint32)
+    cnt = np.array([n, r, int(state["T"])], np.int32)
+    _check(_lib.zsm_cache_import_unit(cache, int(layer), int(b), int(h), _host(K), _host(V),
+                                      _host(score), _host(pos), _host(Kr), _host(Vr), _host(w),
+                                      _host(cnt), _stream(stream)), "zsm_cache_import_unit")
+
+
+def zsm_last_device_status(cache, stream=None) -> int:
+    return int(_lib.zsm_last_device_status(cache, _stream(stream)))
+
+
+def zsm_decode_launch_info(cache, layer):
+    g, b, s = C.c_int32(), C.c_int32(), C.c_int32()
+    _check(_lib.zsm_decode_launch_info(cache, int(layer), C.byref(g), C.byref(b), C.byref(s)),
+           "zsm_decode_launch_info")
+    return g.value, b.value, s.value

@@ -1,0 +1,70 @@
+// Launch interface of the fused decode-step kernel.
+#pragma once
+
+#include "zsm_common.cuh"
+
+namespace zsm {
+
+constexpr int kTileBytes = 16384;      // one ring stage
+constexpr int kMaxConsumerWarps = 16;  // + 1 producer warp
+
+struct DecodeParams {
+    uint8_t *base;               // cache buffer
+    const int32_t *sched_off;    // [grid + 1] first schedule entry of each CTA
+    const UnitDesc *sched_desc;  // unit descriptors in CTA order
+    UnitCounters *counters;      // [n_units]
+    int32_t *status;             // sticky device status
+    const void *q;               // [units][G][d]
+    const void *k_new;           // [units][d]
+    const void *v_new;           // [units][d]
+    void *out;                   // [units][G][d]
+    int32_t *victim_pos;         // [units] or null
+    int32_t *merge_slot;         // [units] or null
+    int32_t unit_base;           // global index of the tensors' first unit
+    int32_t stages;              // ring depth
+    int32_t l_stride;            // floats per query head in the weight array
+    int32_t br_max_pad;          // largest B_r, rounded up to 4
+    float lambda, alpha, scale;
+};
+
+// Shared-memory map of one CTA (byte offsets), computed the same way on host and device.
+struct DecodeSmem {
+    uint32_t ring, bars, flags, probs, qf, kn, vn, w, opart, redf, red64, dots, rows, total;
+};
+
+__host__ __device__ inline DecodeSmem decode_smem_layout(int stages, int G, int D, int row_bytes,
+                                                         int l_stride, int br_max_pad,
+                                                         int consumer_warps) {
+    DecodeSmem L;
+    uint32_t o = 0;
+    auto take = [&](uint32_t bytes) {
+        uint32_t at = o;
+        o += (bytes + 127u) & ~127u;
+        return at;
+    };
+    L.ring = take(static_cast<uint32_t>(stages) * kTileBytes);
+    L.bars = take(static_cast<uint32_t>(stages) * 16u);
+    L.flags = take(64u);
+    L.probs = take(static_cast<uint32_t>(G) * l_stride * 4u);
+    L.qf = take(static_cast<uint32_t>(G) * D * 4u);
+    L.kn = take(static_cast<uint32_t>(row_bytes));
+    L.vn = take(static_cast<uint32_t>(row_bytes));
+    L.w = take(static_cast<uint32_t>(br_max_pad > 0 ? br_max_pad : 4) * 4u);
+    L.opart = take(static_cast<uint32_t>(consumer_warps) * G * D * 4u);
+    L.redf = take(2u * kMaxConsumerWarps * 8u * 4u);
+    L.red64 = take(kMaxConsumerWarps * 16u);
+    L.dots = take(static_cast<uint32_t>(br_max_pad > 0 ? br_max_pad : 4) * 4u);
+    L.rows = take(4u * D * 4u);
+    L.total = o;
+    return L;
+}
+
+// dtype: 0 fp32, 1 fp16, 2 bf16.  Returns a cudaError_t as int; -1: no kernel for the shape.
+int launch_decode_fused(int dtype, int D, int G, const DecodeParams &p, int grid,
+                        int consumer_warps, cudaStream_t stream);
+// Sets the dynamic shared-memory limit of the matching kernel; returns a cudaError_t as int
+// (-1: no kernel) and the CTAs per SM the occupancy calculator allows.
+int prepare_decode_fused(int dtype, int D, int G, int smem_bytes, int threads,
+                         int *max_ctas_per_sm);
+
+}  // namespace zsm

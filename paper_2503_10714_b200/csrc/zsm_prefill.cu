@@ -1,0 +1,545 @@
+// One-shot compression of a prompt's K/V into the per-head budgets.
+//
+//   P1  scores from the prompt's last W queries: causal softmax rows combined by
+//       Eq. (score) unrolled, s_t = (1/G) sum_g sum_tau lambda^(T-1-tau) a_t^(tau)
+//         prefill_logits   scaled, masked q.k into scratch + per-chunk (max, sum exp)
+//         prefill_rowstat  per query row: max and weight/sum
+//         prefill_scores   s_t = sum_rows exp(logit - max) * weight/sum
+//   P2  the latest B_p positions are kept as they are (Sec. 3.2)
+//   P3  prefill_select     of the rest, the B_c highest (score, position) stay: radix
+//                          select of the eviction threshold, then ordered compaction
+//   P4  prefill_merge      evicted tokens, ascending position, fill-or-merge into the
+//                          residual slots (Alg. 1 l.12-16, Eq. (hatr), (kvr))
+//   P5  prefill_gather     survivors' rows, scores and positions into the unit's slots
+#include "zsm_prefill.cuh"
+
+namespace zsm {
+
+namespace {
+
+__device__ __forceinline__ uint32_t order_bits(float s) {
+    // monotone map float -> uint32 (also right for negative inputs)
+    const uint32_t u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// ---------------------------------------------------------------------------
+// P1a: logits of one chunk of prompt positions against every window query.
+// grid (chunks, units), 256 threads: thread (tx, ty) owns positions tx+32i and
+// query rows ty*4+j of the current block of 32 query rows.
+// ---------------------------------------------------------------------------
+constexpr int kQB = 32;  // query rows per pass
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256) prefill_logits_kernel(const PrefillParams p) {
+    using E = Elem<T>;
+    constexpr int CH = kPrefillChunk;
+    constexpr int LD = D + 4;  // padded row, keeps 128-bit shared loads conflict-free
+    extern __shared__ __align__(16) float sm[];
+    float *Ks = sm;            // [CH][LD]
+    float *Qs = sm + CH * LD;  // [kQB][LD]
+
+    const int ul = blockIdx.y;
+    const int b = ul / p.n_kv_heads, h = ul % p.n_kv_heads;
+    const int t0 = blockIdx.x * CH;
+    const int T_len = p.T, W = p.W, G = p.G, GW = p.G * p.W;
+    const int n_chunks = gridDim.x;
+    const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+    const T *Kg = static_cast<const T *>(p.K) + ((size_t)ul * T_len) * D;
+    const int n_q_heads = p.n_kv_heads * G;
+
+    for (int k = tid; k < CH * (D / 4); k += 256) {
+        const int r = k / (D / 4), c = (k % (D / 4)) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t0 + r < T_len) {
+            const T *src = Kg + (size_t)(t0 + r) * D + c;
+            v = make_float4(E::to_float(src[0]), E::to_float(src[1]), E::to_float(src[2]),
+                            E::to_float(src[3]));
+        }
+        *reinterpret_cast<float4 *>(Ks + r * LD + c) = v;
+    }
+    float *logits = reinterpret_cast<float *>(p.ws + p.wl.logits) + (size_t)ul * GW * T_len;
+    float2 *partial = reinterpret_cast<float2 *>(p.ws + p.wl.partial) + (size_t)ul * GW * n_chunks;
+
+    for (int qb = 0; qb < GW; qb += kQB) {
+        __syncthreads();
+        for (int k = tid; k < kQB * (D / 4); k += 256) {
+            const int r = k / (D / 4), c = (k % (D / 4)) * 4;
+            const int gw = qb + r;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (gw < GW) {
+                const int g = gw / W, wq = gw % W;
+                const T *src = static_cast<const T *>(p.Qw) +
+                               (((size_t)b * n_q_heads + h * G + g) * W + wq) * D + c;
+                v = make_float4(E::to_float(src[0]), E::to_float(src[1]), E::to_float(src[2]),
+                                E::to_float(src[3]));
+            }
+            *reinterpret_cast<float4 *>(Qs + r * LD + c) = v;
+        }
+        __syncthreads();
+        float acc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+        for (int dd = 0; dd < D; dd += 4) {
+            float4 a[4], q4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                a[i] = *reinterpret_cast<const float4 *>(Ks + (tx + 32 * i) * LD + dd);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                q4[j] = *reinterpret_cast<const float4 *>(Qs + (ty * 4 + j) * LD + dd);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc[i][j] = fmaf(a[i].x, q4[j].x, acc[i][j]);
+                    acc[i][j] = fmaf(a[i].y, q4[j].y, acc[i][j]);
+                    acc[i][j] = fmaf(a[i].z, q4[j].z, acc[i][j]);
+                    acc[i][j] = fmaf(a[i].w, q4[j].w, acc[i][j]);
+                }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int gw = qb + ty * 4 + j;
+            if (gw >= GW) continue;  // uniform per warp
+            const int tau = T_len - W + (gw % W);  // the query's own position: keys 0..tau
+            float m = -INFINITY;
+            float lg[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int t = t0 + tx + 32 * i;
+                lg[i] = (t < T_len && t <= tau) ? acc[i][j] * p.scale : -INFINITY;
+                if (t < T_len) logits[(size_t)gw * T_len + t] = lg[i];
+                m = fmaxf(m, lg[i]);
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+            float sum = 0.f;
+            if (m > -INFINITY) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sum += expf(lg[i] - m);
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+            if (tx == 0) partial[(size_t)gw * n_chunks + blockIdx.x] = make_float2(m, sum);
+        }
+    }
+}
+
+// P1b: one thread per (unit, query row): fold the chunk partials.
+__global__ void prefill_rowstat_kernel(const PrefillParams p, int n_chunks) {
+    const int GW = p.G * p.W;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= p.units * GW) return;
+    const float2 *part = reinterpret_cast<const float2 *>(p.ws + p.wl.partial) + (size_t)idx * n_chunks;
+    float m = -INFINITY;
+    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, part[c].x);
+    float z = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+        const float2 v = part[c];
+        if (v.x > -INFINITY) z += v.y * expf(v.x - m);
+    }
+    const int wq = idx % p.W;
+    // weight of query position tau = T-W+wq in Eq. (score) unrolled, and the group mean
+    const double coef = pow(static_cast<double>(p.lambda), static_cast<double>(p.W - 1 - wq)) /
+                        static_cast<double>(p.G);
+    reinterpret_cast<float2 *>(p.ws + p.wl.rowstat)[idx] =
+        make_float2(m, static_cast<float>(coef / static_cast<double>(z)));
+}
+
+// P1c: one thread per (unit, position).
+__global__ void prefill_scores_kernel(const PrefillParams p) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int ul = blockIdx.y;
+    if (t >= p.T) return;
+    const int GW = p.G * p.W;
+    const float *logits = reinterpret_cast<const float *>(p.ws + p.wl.logits) + (size_t)ul * GW * p.T;
+    const float2 *rs = reinterpret_cast<const float2 *>(p.ws + p.wl.rowstat) + (size_t)ul * GW;
+    float s = 0.f;
+    for (int gw = 0; gw < GW; ++gw) {
+        const float2 st = __ldg(rs + gw);
+        s = fmaf(expf(logits[(size_t)gw * p.T + t] - st.x), st.y, s);
+    }
+    reinterpret_cast<float *>(p.ws + p.wl.scores)[(size_t)ul * p.T + t] = s;
+}
+
+// ---------------------------------------------------------------------------
+// P2 + P3: one CTA per unit.  Radix select (8 bits per pass, most significant
+// first) of the n_ev-th smallest (score, position) key among the candidates,
+// then two ordered compactions.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) prefill_select_kernel(const PrefillParams p,
+                                                              const float *scores) {
+    __shared__ uint32_t hist[256];
+    __shared__ uint64_t s_prefix;
+    __shared__ uint32_t s_k;
+    __shared__ uint32_t wsum_e[32], wsum_k[32];
+    __shared__ uint32_t base_e, base_k;
+
+    const int ul = blockIdx.x;
+    const UnitDesc d = p.desc[ul];
+    const int T_len = p.T;
+    const int n_prox = min(T_len, d.Bp);
+    const int n_cand = T_len - n_prox;
+    const int n_ev = max(0, n_cand - d.Bc);
+    const float *s = scores + (size_t)ul * T_len;
+    uint8_t *flags = p.ws + p.wl.flags + (size_t)ul * T_len;
+    int32_t *evl = reinterpret_cast<int32_t *>(p.ws + p.wl.evict_list) + (size_t)ul * T_len;
+    int32_t *kpl = reinterpret_cast<int32_t *>(p.ws + p.wl.kept_list) + (size_t)ul * T_len;
+    const int tid = threadIdx.x;
+
+    auto key_of = [&](int t) -> uint64_t {
+        return (static_cast<uint64_t>(order_bits(s[t])) << 32) | static_cast<uint32_t>(t);
+    };
+
+    uint64_t thr = 0;
+    if (n_ev > 0) {
+        if (tid == 0) {
+            s_prefix = 0;
+            s_k = static_cast<uint32_t>(n_ev);
+        }
+        for (int pass = 7; pass >= 0; --pass) {
+            const int shift = pass * 8;
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            const uint64_t prefix = s_prefix;
+            for (int t = tid; t < n_cand; t += blockDim.x) {
+                const uint64_t key = key_of(t);
+                const bool match = (pass == 7) || ((key >> (shift + 8)) == (prefix >> (shift + 8)));
+                if (match) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                uint32_t k = s_k, cum = 0;
+                int dg = 0;
+                for (; dg < 256; ++dg) {
+                    if (cum + hist[dg] >= k) break;
+                    cum += hist[dg];
+                }
+                s_k = k - cum;
+                s_prefix = prefix | (static_cast<uint64_t>(dg) << shift);
+            }
+            __syncthreads();
+        }
+        thr = s_prefix;
+    }
+
+    if (tid == 0) {
+        base_e = 0;
+        base_k = 0;
+    }
+    __syncthreads();
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int t0 = 0; t0 < T_len; t0 += blockDim.x) {
+        const int t = t0 + tid;
+        const bool in = t < T_len;
+        const bool ev = in && n_ev > 0 && t < n_cand && key_of(t) <= thr;
+        const bool kp = in && !ev;
+        if (in) flags[t] = ev ? 1 : 0;
+        const uint32_t be = __ballot_sync(0xffffffffu, ev);
+        const uint32_t bk = __ballot_sync(0xffffffffu, kp);
+        if (lane == 0) {
+            wsum_e[warp] = __popc(be);
+            wsum_k[warp] = __popc(bk);
+        }
+        __syncthreads();
+        uint32_t oe = base_e, ok = base_k;
+        for (int wv = 0; wv < warp; ++wv) {
+            oe += wsum_e[wv];
+            ok += wsum_k[wv];
+        }
+        const uint32_t lt = (1u << lane) - 1u;
+        if (ev) evl[oe + __popc(be & lt)] = t;
+        if (kp) kpl[ok + __popc(bk & lt)] = t;
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t te = 0, tk = 0;
+            for (int wv = 0; wv < (int)(blockDim.x >> 5); ++wv) {
+                te += wsum_e[wv];
+                tk += wsum_k[wv];
+            }
+            base_e += te;
+            base_k += tk;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        int32_t *cnt = reinterpret_cast<int32_t *>(p.ws + p.wl.counts) + ul * 4;
+        cnt[0] = static_cast<int32_t>(base_e);
+        cnt[1] = static_cast<int32_t>(base_k);
+        if (static_cast<int32_t>(base_e) != n_ev) dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 3);
+    }
+    if (p.dbg_evicted) {
+        __syncthreads();
+        for (int t = tid; t < T_len; t += blockDim.x) p.dbg_evicted[(size_t)ul * T_len + t] = flags[t];
+    }
+    if (p.dbg_scores) {
+        for (int t = tid; t < T_len; t += blockDim.x) p.dbg_scores[(size_t)ul * T_len + t] = s[t];
+    }
+}
+
+// ---------------------------------------------------------------------------
+// P4: one CTA per unit walks the evicted tokens in ascending position.  The B_r
+// residual rows live in shared memory as fp32; evicted rows arrive through a small
+// cp.async ring, several tokens ahead of the merge that needs them.
+// ---------------------------------------------------------------------------
+constexpr int kMergeWarps = 8;
+constexpr int kMergePF = 8;     // ring slots
+constexpr int kMergeIB = 512;   // evicted positions staged in shared memory at a time
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kMergeWarps * 32) prefill_merge_kernel(const PrefillParams p) {
+    using E = Elem<T>;
+    constexpr int ROWB = D * (int)sizeof(T);
+    constexpr int CPR = ROWB / 16;  // 16-byte chunks per row
+    constexpr int EPT = D / 32;     // elements per lane
+    static_assert(2 * CPR <= kMergeWarps * 32, "one cp.async per thread covers a K and a V row");
+    extern __shared__ __align__(16) uint8_t smraw[];
+
+    const int ul = blockIdx.x;
+    const UnitDesc d = p.desc[ul];
+    const int Br = d.Br;
+    const int T_len = p.T;
+    const int n_ev = reinterpret_cast<const int32_t *>(p.ws + p.wl.counts)[ul * 4];
+    const int32_t *evl = reinterpret_cast<const int32_t *>(p.ws + p.wl.evict_list) + (size_t)ul * T_len;
+    int32_t *targets = p.dbg_targets ? p.dbg_targets + (size_t)ul * T_len : nullptr;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    if (Br == 0) {
+        if (targets)
+            for (int i = tid; i < n_ev; i += blockDim.x) targets[i] = -1;  // dropped (Sec. 3.2)
+        return;
+    }
+    const int br_pad = (Br + 3) & ~3;
+    float *Kr_s = reinterpret_cast<float *>(smraw);
+    float *Vr_s = Kr_s + (size_t)Br * D;
+    float *dots_s = Vr_s + (size_t)Br * D;
+    uint32_t *w_s = reinterpret_cast<uint32_t *>(dots_s + br_pad);
+    int32_t *idx_s = reinterpret_cast<int32_t *>(w_s + br_pad);         // [kMergeIB + kMergePF]
+    uint8_t *ring = reinterpret_cast<uint8_t *>(idx_s + kMergeIB + kMergePF);  // [PF][2][ROWB]
+
+    const uint8_t *Kg = static_cast<const uint8_t *>(p.K) + (size_t)ul * T_len * ROWB;
+    const uint8_t *Vg = static_cast<const uint8_t *>(p.V) + (size_t)ul * T_len * ROWB;
+
+    // idx_s[j] = evl[i0 + j] for the current block of evicted tokens starting at i0
+    int i0 = 0;
+    auto stage_indices = [&](int start) {
+        for (int j = tid; j < kMergeIB + kMergePF; j += blockDim.x)
+            idx_s[j] = (start + j < n_ev) ? evl[start + j] : 0;
+    };
+    auto issue = [&](int i) {  // fetch evicted token i's rows into ring slot i % PF
+        if (i < n_ev && tid < 2 * CPR) {
+            const int which = tid / CPR, c = tid % CPR;
+            const int t = idx_s[i - i0];
+            const uint8_t *src = (which ? Vg : Kg) + (size_t)t * ROWB + c * 16;
+            cp_async16(ring + ((size_t)(i % kMergePF) * 2 + which) * ROWB + c * 16, src);
+        }
+        cp_async_commit();
+    };
+
+    stage_indices(0);
+    __syncthreads();
+    for (int i = 0; i < kMergePF - 1; ++i) issue(i);
+
+    for (int i = 0; i < n_ev; ++i) {
+        if (i - i0 == kMergeIB) {  // next block of positions (every thread is past iteration i-1)
+            i0 = i;
+            stage_indices(i0);
+            __syncthreads();
+        }
+        issue(i + kMergePF - 1);
+        cp_async_wait<kMergePF - 1>();
+        __syncthreads();  // token i's rows are in the ring for everyone
+        const T *kc_row = reinterpret_cast<const T *>(ring + ((size_t)(i % kMergePF) * 2 + 0) * ROWB);
+        const T *vc_row = reinterpret_cast<const T *>(ring + ((size_t)(i % kMergePF) * 2 + 1) * ROWB);
+        if (i < Br) {
+            // Alg. 1 l.12-13: free slot
+            for (int k = tid; k < D; k += blockDim.x) {
+                Kr_s[(size_t)i * D + k] = E::to_float(kc_row[k]);
+                Vr_s[(size_t)i * D + k] = E::to_float(vc_row[k]);
+            }
+            if (tid == 0) {
+                w_s[i] = 1;
+                if (targets) targets[i] = -2;
+            }
+        } else {
+            float kc[EPT];
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) kc[e] = E::to_float(kc_row[lane * EPT + e]);
+            for (int r = warp; r < Br; r += kMergeWarps) {  // Eq. (hatr)
+                const float *kr = Kr_s + (size_t)r * D + lane * EPT;
+                float acc = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) acc = fmaf(kr[e], kc[e], acc);
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                if (lane == 0) dots_s[r] = acc;
+            }
+            __syncthreads();
+            float bd = -INFINITY;
+            int br = 0x7fffffff;
+            for (int r = lane; r < Br; r += 32) {
+                const float dv = dots_s[r];
+                if (br == 0x7fffffff || dv > bd) {
+                    bd = dv;
+                    br = r;
+                }
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+                const float od = __shfl_xor_sync(0xffffffffu, bd, off);
+                const int orr = __shfl_xor_sync(0xffffffffu, br, off);
+                if (orr != 0x7fffffff && (br == 0x7fffffff || od > bd || (od == bd && orr < br))) {
+                    bd = od;
+                    br = orr;
+                }
+            }
+            if (warp == br % kMergeWarps) {  // Eq. (kvr)
+                const float wr = static_cast<float>(w_s[br]);
+                float *kr = Kr_s + (size_t)br * D + lane * EPT;
+                float *vr = Vr_s + (size_t)br * D + lane * EPT;
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) {
+                    kr[e] = fmaf(wr, kr[e], kc[e]) / (wr + 1.0f);
+                    vr[e] = fmaf(wr, vr[e], E::to_float(vc_row[lane * EPT + e])) / (wr + 1.0f);
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    w_s[br] += 1u;
+                    if (targets) targets[i] = br;
+                }
+            }
+        }
+        __syncthreads();  // rows updated; ring slot i % PF may be refilled
+    }
+    cp_async_wait<0>();
+
+    const int n_res = min(Br, n_ev);
+    float *Kr_g = reinterpret_cast<float *>(p.base + d.kr_off);
+    float *Vr_g = reinterpret_cast<float *>(p.base + d.vr_off);
+    uint32_t *w_g = reinterpret_cast<uint32_t *>(p.base + d.w_off);
+    for (int k = tid; k < n_res * D; k += blockDim.x) {
+        Kr_g[k] = Kr_s[k];
+        Vr_g[k] = Vr_s[k];
+    }
+    for (int k = tid; k < n_res; k += blockDim.x) w_g[k] = w_s[k];
+}
+
+// ---------------------------------------------------------------------------
+// P5: survivors into the unit's slots, ascending position; one warp per row.
+// ---------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(256) prefill_gather_kernel(const PrefillParams p, const float *scores) {
+    constexpr int ROWB = D * (int)sizeof(T);
+    constexpr int CPR = ROWB / 16;
+    const int ul = blockIdx.y;
+    const UnitDesc d = p.desc[ul];
+    const int T_len = p.T;
+    const int32_t *cnt = reinterpret_cast<const int32_t *>(p.ws + p.wl.counts) + ul * 4;
+    const int n_ev = cnt[0], n_kept = cnt[1];
+    const int cap = d.Bp + d.Bc;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (n_kept > cap) dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 4);
+        UnitCounters c;
+        c.n_live = min(n_kept, cap);
+        c.n_res = min(d.Br, n_ev);
+        c.T = T_len;
+        c.pad = 0;
+        p.counters[d.unit] = c;
+    }
+    const int row = blockIdx.x * 8 + warp;
+    if (row >= min(n_kept, cap)) return;
+    const int t = reinterpret_cast<const int32_t *>(p.ws + p.wl.kept_list)[(size_t)ul * T_len + row];
+    const uint4 *ks = reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(p.K) + ((size_t)ul * T_len + t) * ROWB);
+    const uint4 *vs = reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(p.V) + ((size_t)ul * T_len + t) * ROWB);
+    uint4 *kd = reinterpret_cast<uint4 *>(p.base + d.k_off + (size_t)row * ROWB);
+    uint4 *vd = reinterpret_cast<uint4 *>(p.base + d.v_off + (size_t)row * ROWB);
+    for (int c = lane; c < CPR; c += 32) {
+        kd[c] = ks[c];
+        vd[c] = vs[c];
+    }
+    if (lane == 0) {
+        reinterpret_cast<float *>(p.base + d.score_off)[row] = scores[(size_t)ul * T_len + t];
+        reinterpret_cast<int32_t *>(p.base + d.pos_off)[row] = t;
+    }
+}
+
+template <int D>
+size_t merge_smem_bytes(int Br, int row_bytes) {
+    const int br_pad = (Br + 3) & ~3;
+    return (size_t)Br * D * 8 + (size_t)br_pad * 8 + (size_t)(kMergeIB + kMergePF) * 4 +
+           (size_t)kMergePF * 2 * row_bytes;
+}
+
+template <typename T, int D>
+int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
+    const int n_chunks = (p.T + kPrefillChunk - 1) / kPrefillChunk;
+    const float *scores = p.scores_in;
+    if (p.Qw) {
+        const size_t sm = (size_t)(kPrefillChunk + kQB) * (D + 4) * 4;
+        prefill_logits_kernel<T, D><<<dim3(n_chunks, p.units), 256, sm, stream>>>(p);
+        const int rows = p.units * p.G * p.W;
+        prefill_rowstat_kernel<<<(rows + 127) / 128, 128, 0, stream>>>(p, n_chunks);
+        prefill_scores_kernel<<<dim3((p.T + 255) / 256, p.units), 256, 0, stream>>>(p);
+        scores = reinterpret_cast<const float *>(p.ws + p.wl.scores);
+    }
+    prefill_select_kernel<<<p.units, 1024, 0, stream>>>(p, scores);
+    prefill_merge_kernel<T, D><<<p.units, kMergeWarps * 32,
+                                 merge_smem_bytes<D>(max_br, D * (int)sizeof(T)), stream>>>(p);
+    // the largest unit bounds the gather grid; rows past a unit's survivors return at once
+    const int max_rows = p.max_cap < p.T ? p.max_cap : p.T;
+    prefill_gather_kernel<T, D><<<dim3((max_rows + 7) / 8, p.units), 256, 0, stream>>>(p, scores);
+    return static_cast<int>(cudaGetLastError());
+}
+
+template <typename T, int D>
+int prepare_all() {
+    cudaError_t e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)((kPrefillChunk + kQB) * (D + 4) * 4));
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = cudaFuncSetAttribute(prefill_merge_kernel<T, D>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)merge_smem_bytes<D>(prefill_max_residual(D), D * (int)sizeof(T)));
+    return static_cast<int>(e);
+}
+
+}  // namespace
+
+int prefill_max_residual(int D) { return (192 * 1024) / (D * 8); }
+
+int launch_prefill(int dtype, int D, const PrefillParams &p, int max_br, cudaStream_t stream) {
+    if (dtype == 0 && D == 64) return launch_all<float, 64>(p, max_br, stream);
+    if (dtype == 0 && D == 128) return launch_all<float, 128>(p, max_br, stream);
+    if (dtype == 1 && D == 64) return launch_all<__half, 64>(p, max_br, stream);
+    if (dtype == 1 && D == 128) return launch_all<__half, 128>(p, max_br, stream);
+    if (dtype == 2 && D == 64) return launch_all<__nv_bfloat16, 64>(p, max_br, stream);
+    if (dtype == 2 && D == 128) return launch_all<__nv_bfloat16, 128>(p, max_br, stream);
+    return -1;
+}
+
+int prepare_prefill(int dtype, int D) {
+    if (dtype == 0 && D == 64) return prepare_all<float, 64>();
+    if (dtype == 0 && D == 128) return prepare_all<float, 128>();
+    if (dtype == 1 && D == 64) return prepare_all<__half, 64>();
+    if (dtype == 1 && D == 128) return prepare_all<__half, 128>();
+    if (dtype == 2 && D == 64) return prepare_all<__nv_bfloat16, 64>();
+    if (dtype == 2 && D == 128) return prepare_all<__nv_bfloat16, 128>();
+    return -1;
+}
+
+}  // namespace zsm

@@ -1,0 +1,232 @@
+"""GPU parity of the fused decode step against the oracle, element by element, through
+the C ABI.  Small and medium shapes that span several tiles and ragged tails; the
+degenerate budgets the method has; both launch shapes (all layers / one layer)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from harness import (GpuCache, ParityStats, f64, oracle_step_check, oracle_unit_for, split_budgets,
+                     state_check)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def zb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2503_10714_b200 import binding
+    return binding
+
+
+def run_decode(zb, oracle, w, bp, bc, br, steps, layer_mode=-1, check_state_every=25, alpha=1.0,
+               lam=0.98, units=None, **tune):
+    cache = GpuCache(zb, w, bp, bc, br, lam=lam, alpha=alpha, **tune)
+    stats = ParityStats()
+    try:
+        if units is None:
+            units = [(l, b, h) for l in range(w.n_layers) for b in range(w.batch)
+                     for h in range(w.n_kv_heads)]
+        orc = {u: oracle_unit_for(oracle, cache, u[0], u[2]) for u in units}
+        G = w.group
+        for step in range(steps):
+            q, k, v = wl.decode_inputs(w, step)
+            out, vic, slot = cache.decode(q.cuda(), k.cuda(), v.cuda(), layer=layer_mode)
+            out_h, vic_h, slot_h = f64(out), vic.cpu().numpy(), slot.cpu().numpy()
+            q64, k64, v64 = f64(q), f64(k), f64(v)
+            for (l, b, h), unit in orc.items():
+                oracle_step_check(unit, q64[l, b, h * G:(h + 1) * G], k64[l, b, h], v64[l, b, h],
+                                  out_h[l, b, h * G:(h + 1) * G], vic_h[l, b, h], slot_h[l, b, h],
+                                  w.dtype, stats, tag=f"step {step} unit {(l, b, h)}")
+            if (step + 1) % check_state_every == 0 or step == steps - 1:
+                for (l, b, h), unit in orc.items():
+                    state_check(unit, cache.export(l, b, h), stats, tag=f"step {step} unit {(l, b, h)}")
+        assert cache.status() == 0
+    finally:
+        cache.close()
+    assert stats.exact_tie_breaches == 0
+    return stats
+
+
+SMALL = wl.Workload("small", 2, 2, 2, 2, 64, "f32", 0, 0, 0, None, 11)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("head_dim", [64, 128])
+@pytest.mark.parametrize("group", [1, 4])
+def test_decode_from_empty_all_kernel_variants(zb, oracle, dtype, head_dim, group):
+    """Every (dtype, head_dim, group) kernel: fill, first evictions, residual fill, merges."""
+    w = SMALL.replace(dtype=dtype, head_dim=head_dim, n_q_heads=2 * group)
+    bp = np.array([[6, 9], [4, 20]])
+    bc = np.array([[7, 30], [5, 11]])
+    br = np.array([[2, 3], [1, 5]])
+    stats = run_decode(zb, oracle, w, bp, bc, br, steps=90)
+    assert stats.selections > 200 and stats.merges > 150
+
+
+@pytest.mark.parametrize("budgets", [(0, 5, 3), (5, 0, 2), (4, 6, 0), (1, 1, 1), (0, 1, 0), (1, 0, 1)])
+def test_degenerate_budgets(zb, oracle, budgets):
+    """B_p = 0 (the new token competes at once), B_c = 0 (whatever leaves proximity is evicted),
+    B_r = 0 (pure eviction) and the smallest caches."""
+    w = SMALL.replace(dtype="f16", head_dim=128, n_layers=1)
+    bp, bc, br = (np.full((1, 2), x) for x in budgets)
+    run_decode(zb, oracle, w, bp, bc, br, steps=40, check_state_every=5)
+
+
+@pytest.mark.parametrize("alpha,lam", [(0.0, 0.98), (0.5, 0.5), (1.0, 0.0), (1.0, 1.0)])
+def test_alpha_and_lambda_range(zb, oracle, alpha, lam):
+    w = SMALL.replace(dtype="f16", head_dim=128, n_layers=1)
+    run_decode(zb, oracle, w, np.full((1, 2), 5), np.full((1, 2), 6), np.full((1, 2), 2), steps=50,
+               alpha=alpha, lam=lam)
+
+
+@pytest.mark.parametrize("layer_mode", [-1, "each"])
+def test_multi_tile_ragged_units(zb, oracle, layer_mode):
+    """Slot pools that span several 16 KiB tiles with a ragged last tile, ragged per-head
+    budgets, residual pools larger than one tile row group; both launch shapes."""
+    w = wl.Workload("ragged", 2, 2, 8, 4, 128, "f16", 0, 0, 0, None, 12)
+    rs = np.random.RandomState(5)
+    tot = rs.randint(70, 260, size=(2, 4))
+    bp, bc, br = split_budgets(zb, tot)
+    br[0, 1], br[1, 2] = 37, 0
+    stats = run_decode(zb, oracle, w, bp, bc, br, steps=300, layer_mode=layer_mode,
+                       check_state_every=100)
+    assert stats.selections > 1000
+
+
+def test_budget_at_least_context_is_full_attention(zb):
+    """Invariant: while nothing is evicted the output is plain softmax attention over the
+    whole history (checked against torch SDPA in fp64 on the CPU, not against the oracle)."""
+    w = wl.Workload("full", 1, 2, 4, 2, 128, "f16", 0, 0, 0, None, 13)
+    steps = 150
+    cache = GpuCache(zb, w, np.full((1, 2), 40), np.full((1, 2), steps), np.full((1, 2), 3))
+    try:
+        qs, ks, vs = [], [], []
+        for step in range(steps):
+            q, k, v = wl.decode_inputs(w, step)
+            out, vic, _ = cache.decode(q.cuda(), k.cuda(), v.cuda())
+            qs.append(q[0]), ks.append(k[0]), vs.append(v[0])
+            K = torch.stack(ks, dim=2).double().repeat_interleave(w.group, dim=1)   # [b,Hq,t,d]
+            V = torch.stack(vs, dim=2).double().repeat_interleave(w.group, dim=1)
+            ref = torch.nn.functional.scaled_dot_product_attention(q[0].double()[:, :, None, :], K, V)
+            torch.testing.assert_close(out[0].cpu().double(), ref[:, :, 0, :], atol=2e-3, rtol=1e-2)
+            assert (vic.cpu() == -1).all()
+        assert cache.status() == 0
+    finally:
+        cache.close()
+
+
+def test_exact_ties_resolve_by_position(zb):
+    """Bit-identical tokens give bit-identical scores on the GPU too: the evicted one must be
+    the lowest position among the minima (lam = 0, as in the oracle's pin)."""
+    w = wl.Workload("ties", 1, 1, 1, 1, 64, "f32", 0, 0, 0, None, 14)
+    cache = GpuCache(zb, w, [[1]], [[2]], [[0]], lam=0.0)
+    try:
+        def tok(x):
+            t = torch.zeros(1, 1, 1, 64)
+            t[..., 0] = x
+            return t.cuda()
+        q, ones = tok(1.0), torch.ones(1, 1, 1, 64).cuda()
+        seq = [1.0, 1.0, 5.0, 5.0, 5.0]
+        victims = []
+        for x in seq:
+            _, vic, _ = cache.decode(q, tok(x), ones)
+            victims.append(int(vic.cpu()[0, 0, 0]))
+        assert victims == [-1, -1, -1, 0, 1]
+    finally:
+        cache.close()
+
+
+def test_decode_from_imported_large_state(zb, oracle):
+    """A unit larger than one (score, pos) tile (2048 entries) and a residual pool of 60
+    slots: state built by the oracle's prompt pass, imported through the C ABI, then decoded
+    on both sides."""
+    w = wl.Workload("large", 1, 1, 2, 1, 128, "bf16", 0, 0, 0, None, 15)
+    bp, bc, br = 1100, 1250, 60
+    T = 3000
+    g = torch.Generator().manual_seed(3)
+    K = torch.randn(T, 128, generator=g).to(torch.bfloat16)
+    V = torch.randn(T, 128, generator=g).to(torch.bfloat16)
+    scores = torch.rand(T, generator=g).numpy().astype(np.float32) + 1e-3
+    cache = GpuCache(zb, w, [[bp]], [[bc]], [[br]])
+    stats = ParityStats()
+    try:
+        unit = oracle_unit_for(oracle, cache, 0, 0)
+        unit.prefill_compress(f64(K), f64(V), scores=scores)
+        pos, sc, Kt, Vt = unit.tokens()
+        Kr, Vr, wr = unit.residual()
+        state = dict(K=Kt, V=Vt, score=sc, pos=pos, Kr=Kr, Vr=Vr, w=wr, n_live=len(pos),
+                     n_res=len(wr), T=T)
+        zb.zsm_cache_import_unit(cache.h, 0, 0, 0, 128, state)
+        state_check(unit, cache.export(0, 0, 0), stats, tag="after import")
+        for step in range(60):
+            q, k, v = wl.decode_inputs(w, step)
+            out, vic, slot = cache.decode(q.cuda(), k.cuda(), v.cuda())
+            oracle_step_check(unit, f64(q)[0, 0], f64(k)[0, 0, 0], f64(v)[0, 0, 0], f64(out)[0, 0],
+                              int(vic.cpu()[0, 0, 0]), int(slot.cpu()[0, 0, 0]), w.dtype, stats,
+                              tag=f"step {step}")
+        state_check(unit, cache.export(0, 0, 0), stats, tag="end")
+        assert cache.status() == 0 and stats.merges == 60
+    finally:
+        cache.close()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point(zb):
+    """zsm_decode_step_host = copies in, the same kernel, copy out."""
+    w = wl.Workload("host", 2, 2, 4, 2, 128, "f16", 0, 0, 0, None, 16)
+    mk = lambda: GpuCache(zb, w, np.full((2, 2), 8), np.full((2, 2), 9), np.full((2, 2), 2))
+    a, b = mk(), mk()
+    try:
+        staging = torch.empty(zb.zsm_decode_staging_bytes(b.h, -1), dtype=torch.uint8, device="cuda")
+        for step in range(40):
+            q, k, v = wl.decode_inputs(w, step)
+            out, _, _ = a.decode(q.cuda(), k.cuda(), v.cuda())
+            qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+            oh = torch.empty_like(qh).pin_memory()
+            zb.zsm_decode_step_host(b.h, -1, qh, kh, vh, oh, staging)
+            assert torch.equal(out.cpu(), oh)
+        assert a.status() == 0 and b.status() == 0
+    finally:
+        a.close(), b.close()
+
+
+def test_runs_are_bitwise_reproducible(zb):
+    w = wl.Workload("repro", 2, 2, 8, 2, 128, "bf16", 0, 0, 0, None, 17)
+    outs = []
+    for _ in range(2):
+        c = GpuCache(zb, w, np.full((2, 2), 20), np.full((2, 2), 90), np.full((2, 2), 4))
+        try:
+            acc = []
+            for step in range(150):
+                q, k, v = wl.decode_inputs(w, step)
+                out, vic, slot = c.decode(q.cuda(), k.cuda(), v.cuda())
+                acc.append((out.clone(), vic.clone(), slot.clone()))
+            outs.append(acc)
+        finally:
+            c.close()
+    for (o1, v1, s1), (o2, v2, s2) in zip(*outs):
+        assert torch.equal(o1, o2) and torch.equal(v1, v2) and torch.equal(s1, s2)
+
+
+def test_argument_errors_reach_the_caller(zb):
+    w = SMALL.replace(dtype="f16", head_dim=128)
+    c = GpuCache(zb, w, np.full((2, 2), 4), np.full((2, 2), 4), np.full((2, 2), 1))
+    try:
+        q, k, v = (t.cuda() for t in wl.decode_inputs(w, 0))
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_decode_step(c.h, 7, q, k, v, c.out_all)
+        assert e.value.status == zb.ZSM_ERR_INVALID_ARG
+        with pytest.raises(zb.ZsmError):
+            zb.zsm_decode_step(c.h, -1, q.view(-1)[1:], k, v, c.out_all)   # misaligned pointer
+        small = torch.empty(16, dtype=torch.uint8, device="cuda")
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_cache_create(c.cfg, small)
+        assert e.value.status in (zb.ZSM_ERR_BUFFER_TOO_SMALL, zb.ZSM_ERR_INVALID_ARG)
+        bad = zb.make_config(1, 1, 3, 1, 128, "f16", [4], [4], [1])      # group size 3
+        buf = torch.empty(zb.zsm_cache_bytes(bad), dtype=torch.uint8, device="cuda")
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_cache_create(bad, buf)
+        assert e.value.status == zb.ZSM_ERR_UNSUPPORTED
+    finally:
+        c.close()
