@@ -1,0 +1,142 @@
+"""GPU parity of the one-shot prompt compression and of prompt pass + decode end to end
+(workloads c1 and c2 in full) against the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from harness import (GpuCache, ParityStats, f64, oracle_step_check, prefill_check, split_budgets,
+                     state_check)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def zb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2503_10714_b200 import binding
+    return binding
+
+
+def prefill_all_units(zb, oracle, w, cache, layer, stats, scores=None):
+    K, V, Qw = wl.prompt(w, layer)
+    if scores is None:
+        dbg = cache.prefill(layer, K.cuda(), V.cuda(), Qw.cuda())
+    else:
+        dbg = cache.prefill(layer, K.cuda(), V.cuda(), None, scores.cuda())
+    units = {}
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            units[(layer, b, h)] = prefill_check(
+                oracle, cache, layer, b, h, K, V, Qw, dbg, stats,
+                scores_given=None if scores is None else scores[b, h].numpy(),
+                tag=f"prompt pass unit {(layer, b, h)}")
+    return units
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("head_dim,group", [(64, 1), (128, 1), (128, 4), (64, 2)])
+def test_prompt_pass_all_kernel_variants(zb, oracle, dtype, head_dim, group):
+    """Scores, selection, merge chain and gathered state for every kernel variant; prompt of
+    several score chunks with a ragged tail; ragged per-head budgets."""
+    w = wl.Workload("pp", 2, 2, 2 * group, 2, head_dim, dtype, 700, 0, 24, None, 21)
+    bp = np.array([[16, 40], [8, 33]])
+    bc = np.array([[20, 61], [9, 70]])
+    br = np.array([[2, 5], [1, 9]])
+    cache = GpuCache(zb, w, bp, bc, br)
+    stats = ParityStats()
+    try:
+        for layer in range(w.n_layers):
+            prefill_all_units(zb, oracle, w, cache, layer, stats)
+        assert cache.status() == 0
+    finally:
+        cache.close()
+    assert stats.selections > 4000 and stats.merges > 3500
+
+
+@pytest.mark.parametrize("T,window", [(5, 5), (30, 8), (48, 48), (129, 1), (300, 300)])
+def test_prompt_lengths_around_the_budgets(zb, oracle, T, window):
+    """Prompts shorter than B_p, shorter than B_p + B_c (nothing evicted), barely longer
+    (residual slots only partly filled), and a full-history window (W = T)."""
+    w = wl.Workload("len", 1, 1, 2, 2, 128, "f16", T, 0, window, None, 22)
+    cache = GpuCache(zb, w, [[10, 20]], [[25, 100]], [[4, 40]])
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats)
+        assert cache.status() == 0
+    finally:
+        cache.close()
+
+
+@pytest.mark.parametrize("budgets", [(0, 12, 2), (10, 0, 4), (6, 9, 0), (1, 1, 1)])
+def test_prompt_pass_degenerate_budgets(zb, oracle, budgets):
+    w = wl.Workload("deg", 1, 2, 2, 1, 64, "bf16", 200, 0, 16, None, 23)
+    cache = GpuCache(zb, w, [[budgets[0]]], [[budgets[1]]], [[budgets[2]]])
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats)
+    finally:
+        cache.close()
+
+
+def test_supplied_scores_with_exact_ties(zb, oracle):
+    """Scores given by the caller, drawn from four values only: the selection is decided by
+    the position rule almost everywhere and must match the oracle bit for bit (no near tie
+    can exist between distinct values this far apart)."""
+    w = wl.Workload("ties", 1, 2, 2, 2, 128, "f16", 1000, 0, 0, None, 24)
+    g = torch.Generator().manual_seed(1)
+    scores = torch.randint(1, 5, (2, 2, 1000), generator=g).float() * 0.25
+    cache = GpuCache(zb, w, [[50, 64]], [[70, 300]], [[3, 12]])
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats, scores=scores)
+        assert stats.victim_near_ties == 0
+    finally:
+        cache.close()
+
+
+def pipeline(zb, oracle, w, layer_mode=-1, check_state_every=64):
+    """Prompt pass for every layer, then every decode step, every unit checked at every step."""
+    bp, bc, br = split_budgets(zb, wl.head_budgets(w))
+    cache = GpuCache(zb, w, bp, bc, br)
+    stats = ParityStats()
+    try:
+        units = {}
+        for layer in range(w.n_layers):
+            units.update(prefill_all_units(zb, oracle, w, cache, layer, stats))
+        G = w.group
+        for step in range(w.decode_steps):
+            q, k, v = wl.decode_inputs(w, step)
+            out, vic, slot = cache.decode(q.cuda(), k.cuda(), v.cuda(), layer=layer_mode)
+            out_h, vic_h, slot_h = f64(out), vic.cpu().numpy(), slot.cpu().numpy()
+            q64, k64, v64 = f64(q), f64(k), f64(v)
+            for (l, b, h), unit in units.items():
+                oracle_step_check(unit, q64[l, b, h * G:(h + 1) * G], k64[l, b, h], v64[l, b, h],
+                                  out_h[l, b, h * G:(h + 1) * G], vic_h[l, b, h], slot_h[l, b, h],
+                                  w.dtype, stats, tag=f"{w.name} step {step} unit {(l, b, h)}")
+            if (step + 1) % check_state_every == 0 or step == w.decode_steps - 1:
+                for (l, b, h), unit in units.items():
+                    state_check(unit, cache.export(l, b, h), stats, tag=f"{w.name} step {step}")
+        assert cache.status() == 0
+    finally:
+        cache.close()
+    assert stats.exact_tie_breaches == 0
+    return stats
+
+
+def test_workload_c1_full(zb, oracle):
+    """c1: 1 layer, 4 heads, d 64, fp32, prompt 512 scored with its full history, budget 64,
+    64 decode steps: every unit, every step."""
+    stats = pipeline(zb, oracle, wl.C1)
+    assert stats.steps == 4 * 64 and stats.merges >= 4 * 64
+    print("c1", stats)
+
+
+def test_workload_c2_full(zb, oracle):
+    """c2: LLaMA2-7B layer shape, fp16, prompt 4096, budget 205, 256 decode steps: every
+    unit, every step; expected near-tie events: none or a handful."""
+    stats = pipeline(zb, oracle, wl.C2)
+    assert stats.steps == 32 * 256
+    assert stats.victim_near_ties + stats.merge_near_ties <= 64
+    print("c2", stats)
