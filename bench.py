@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Decode-step throughput of the compressed-KV cache path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload NAME]
+
+One step = one fused decode launch over every layer of the workload (score update,
+eviction, residual merge, compensated attention, insertion), on a cache produced by the
+real prompt-compression pass.  Default workload: LLaMA2-7B shape, batch 1, 54 000-token
+prompt, 5 % budget (2 700 slots per head, 1 024 units, 1.45 GB streamed per step --
+far larger than L2, so no flush is needed between steps).
+
+N > 1 (torchrun): every rank runs the same workload on its own sequence (weak scaling,
+no data-path collective); value = tokens of all ranks / max-over-ranks device time.
+
+--impl reference times the CPU oracle (the only other implementation of this path that
+exists) on a bounded sample of the same workload, rank 0 only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def recorded_traffic(name):
+    """DRAM bytes per launch from the committed ncu summary of this workload, if any."""
+    path = os.path.join(ROOT, "profiles", "decode_fused_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(name)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake"}
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                mask = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def __enter__(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def algorithmic_bytes(w, bp, bc, br, n_live, n_res):
+    """Bytes one decode launch must move: every live slot's K and V row once, its score read
+    and written, its position read; every merged slot's fp32 K and V row and count; per unit
+    q, k_new, v_new in, out, the inserted rows and the merged rows out."""
+    e = 4 if w.dtype == "f32" else 2
+    row = w.head_dim * e
+    G = w.group
+    per_unit_fixed = G * row + 2 * row + G * row + 2 * row + 2 * w.head_dim * 4 + 16
+    total = 0
+    for l in range(w.n_layers):
+        for h in range(w.n_kv_heads):
+            total += w.batch * (n_live[l, h] * (2 * row + 12) + n_res[l, h] * (2 * w.head_dim * 4 + 4)
+                                + per_unit_fixed)
+    return int(total)
+
+
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return world, rank, local
+
+
+def max_over_ranks(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda" if torch.cuda.is_available() else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ----------------------------------------------------------------------------- oracle leg
+def oracle_sample(w, K, V, Qw, bp, bc, br, steps, layer=0):
+    """Times the oracle, as it stands, on one layer's units: state from its own prompt pass
+    (untimed), then `steps` decode steps over those units with OpenMP.  Returns
+    (seconds per sampled step, units sampled, threads used)."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    from oracle import zsm_oracle as zo
+    zo.build()
+    G = w.group
+    units = []
+    jobs = [(b, h) for b in range(w.batch) for h in range(w.n_kv_heads)]
+
+    def make(job):
+        b, h = job
+        u = zo.Unit(w.head_dim, G, int(bp[layer, h]), int(bc[layer, h]), int(br[layer, h]),
+                    lam=float(np.float32(0.98)), alpha=1.0)
+        u.prefill_compress(K[b, h].double().numpy(), V[b, h].double().numpy(),
+                           Qw=Qw[b, h * G:(h + 1) * G].double().numpy())
+        return u
+    with ThreadPoolExecutor(max_workers=os.cpu_count() or 1) as ex:
+        units = list(ex.map(make, jobs))
+    qs, ks, vs = [], [], []
+    for step in range(steps):
+        q, k, v = wl.decode_inputs(w.replace(n_layers=1), step)
+        qs.append(q[0].double().numpy().reshape(len(jobs), G, w.head_dim))
+        ks.append(k[0].double().numpy().reshape(len(jobs), w.head_dim))
+        vs.append(v[0].double().numpy().reshape(len(jobs), w.head_dim))
+    threads = 1
+    t0 = time.perf_counter()
+    for step in range(steps):
+        _, threads = zo.decode_step_batch(units, qs[step], ks[step], vs[step])
+    dt = (time.perf_counter() - t0) / steps
+    for u in units:
+        u.close()
+    return dt, len(jobs), threads
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="zsm", choices=["zsm", "reference"])
+    ap.add_argument("--workload", default="c4_54k_5pct", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=200)
+    ap.add_argument("--cpu-steps", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--consumer-warps", type=int, default=0)
+    args = ap.parse_args()
+    world, rank, local = dist_setup(args.gpus)
+    w0 = wl.WORKLOADS[args.workload]
+    W = max(3, args.warmup)
+    K = max(1, args.steps)
+
+    w = w0.replace(seed=w0.seed + 1000 * rank)  # every rank its own sequence
+    from paper_2503_10714_b200 import binding as zb
+    totals = wl.head_budgets(w)
+    bp = np.zeros_like(totals)
+    bc = np.zeros_like(totals)
+    br = np.zeros_like(totals)
+    for idx in np.ndindex(totals.shape):
+        bp[idx], bc[idx], br[idx] = zb.zsm_split_budget(int(totals[idx]))
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    stream = torch.cuda.current_stream()
+    cfg = zb.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, bp,
+                         bc, br, tune_stages=args.stages, tune_ctas_per_sm=args.ctas_per_sm,
+                         tune_consumer_warps=args.consumer_warps)
+    buf = torch.empty(zb.zsm_cache_bytes(cfg), dtype=torch.uint8, device=dev)
+    cache = zb.zsm_cache_create(cfg, buf)
+
+    # ---- prompt pass (real kernels; timed separately, not part of the decode metric) ----
+    u = wl.directions(w, dev)
+    ws = torch.empty(zb.zsm_prefill_workspace_bytes(cache, w.prompt_len, w.window),
+                     dtype=torch.uint8, device=dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    prefill_ms = 0.0
+    sample_prompt = None
+    for layer in range(w.n_layers):
+        Kp, Vp, Qw = wl.prompt(w, layer, dev, u)
+        ev0.record(stream)
+        zb.zsm_prefill_compress(cache, layer, Kp, Vp, Qw, None, w.prompt_len, w.window, ws)
+        ev1.record(stream)
+        ev1.synchronize()
+        prefill_ms += ev0.elapsed_time(ev1)
+        if layer == 0 and rank == 0 and world == 1 and not args.no_cpu_baseline:
+            sample_prompt = (Kp.cpu(), Vp.cpu(), Qw.cpu())
+        del Kp, Vp, Qw
+    del ws
+    if zb.zsm_last_device_status(cache) != 0:
+        raise RuntimeError("device status after the prompt pass is not OK")
+
+    # ---- decode inputs for every step, resident in HBM before timing starts ----
+    n_steps_total = W + K
+    qs = torch.empty(n_steps_total, w.n_layers, w.batch, w.n_q_heads, w.head_dim,
+                     dtype=w.torch_dtype, device=dev)
+    ks = torch.empty(n_steps_total, w.n_layers, w.batch, w.n_kv_heads, w.head_dim,
+                     dtype=w.torch_dtype, device=dev)
+    vs = torch.empty_like(ks)
+    for s in range(n_steps_total):
+        qs[s], ks[s], vs[s] = wl.decode_inputs(w, s, dev, u)
+    out = torch.empty_like(qs[0])
+    for s in range(W):
+        zb.zsm_decode_step(cache, -1, qs[s], ks[s], vs[s], out)
+    torch.cuda.synchronize()
+    barrier(world)
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clocks:
+        ev0.record(stream)
+        for s in range(W, W + K):
+            zb.zsm_decode_step(cache, -1, qs[s], ks[s], vs[s], out)
+        ev1.record(stream)
+        ev1.synchronize()
+    torch.cuda.synchronize()
+    barrier(world)
+    ms_local = ev0.elapsed_time(ev1)
+    ms_total = max_over_ranks(ms_local, world)
+    ms_per_step = ms_total / K
+    if zb.zsm_last_device_status(cache) != 0:
+        raise RuntimeError("device status after the timed region is not OK")
+
+    # ---- the same metric through host buffers (copies inside the timed region) ----
+    Ke = max(1, min(args.e2e_steps, K))
+    staging = torch.empty(zb.zsm_decode_staging_bytes(cache, -1), dtype=torch.uint8, device=dev)
+    qh = [qs[W + s].cpu().pin_memory() for s in range(Ke)]
+    kh = [ks[W + s].cpu().pin_memory() for s in range(Ke)]
+    vh = [vs[W + s].cpu().pin_memory() for s in range(Ke)]
+    oh = torch.empty_like(qh[0]).pin_memory()
+    for s in range(3):
+        zb.zsm_decode_step_host(cache, -1, qh[s], kh[s], vh[s], oh, staging)
+    torch.cuda.synchronize()
+    barrier(world)
+    t0 = time.perf_counter()
+    for s in range(Ke):
+        zb.zsm_decode_step_host(cache, -1, qh[s], kh[s], vh[s], oh, staging)
+    torch.cuda.synchronize()
+    e2e_s = max_over_ranks(time.perf_counter() - t0, world)
+    h2d = qh[0].numel() * qh[0].element_size() + 2 * kh[0].numel() * kh[0].element_size()
+    d2h = oh.numel() * oh.element_size()
+
+    if rank != 0:
+        zb.zsm_cache_free(cache)
+        return
+
+    # ---- roofline of the dominant (only) kernel of the timed region ----
+    n_live = (bp + bc).astype(np.int64)      # every unit is full after a 54k prompt
+    n_res = br.astype(np.int64)
+    n_live = np.minimum(n_live, w.prompt_len + W)
+    abytes = algorithmic_bytes(w, bp, bc, br, n_live, n_res)
+    peak, peak_kind = measured_peak()
+    achieved = abytes / (ms_local / K * 1e-3) / 1e9
+    grid, block, smem = zb.zsm_decode_launch_info(cache, -1)
+    line = {
+        "metric": "decode tokens/s with ZSMerge cache update",
+        "value": world * w.batch * K / (ms_total * 1e-3),
+        "unit": "tokens/s",
+        "n_gpus": world,
+        "steps": K,
+        "warmup": W,
+        "ms_per_step": ms_per_step,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": w.dtype,
+        "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch,
+                   "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                   "prompt_len": w.prompt_len, "slots_per_head": int(totals.mean()),
+                   "launch": "one fused kernel over all layers per step",
+                   "grid": grid, "block": block, "smem_bytes": smem,
+                   "l2": "inputs larger than L2 (%.2f GB streamed per step)" % (abytes / 1e9)},
+        "clocks": clocks.summary(),
+        "e2e": {"value": world * w.batch * Ke / e2e_s, "unit": "tokens/s",
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": Ke},
+        "gpu_launches": K,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_kind,
+                     "algorithmic_bytes_per_launch": abytes,
+                     "traffic": recorded_traffic(w.name)},
+        "prompt_pass": {"ms_total": prefill_ms, "ms_per_layer": prefill_ms / w.n_layers,
+                        "window": w.window},
+    }
+    if world == 1 and not args.no_cpu_baseline and sample_prompt is not None:
+        dt, n_sampled, threads = oracle_sample(w, *sample_prompt, bp, bc, br, args.cpu_steps)
+        n_units = w.n_layers * w.batch * w.n_kv_heads
+        line["cpu_baseline"] = {
+            "value": w.batch / (dt * n_units / n_sampled), "unit": "tokens/s", "cores": threads,
+            "kind": "oracle",
+            "sample": "%d of %d units (layer 0) x %d decode steps, scaled by units" % (
+                n_sampled, n_units, args.cpu_steps)}
+    zb.zsm_cache_free(cache)
+    print(json.dumps(line))
+
+
+def main_reference():
+    """--impl reference: the oracle on the machine's host cores, a bounded sample per step."""
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="reference")
+    ap.add_argument("--workload", default="c4_54k_5pct", choices=sorted(wl.WORKLOADS))
+    args, _ = ap.parse_known_args()
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    w = wl.WORKLOADS[args.workload]
+    from oracle import zsm_oracle as zo
+    totals = wl.head_budgets(w)
+    bp = np.zeros_like(totals)
+    bc = np.zeros_like(totals)
+    br = np.zeros_like(totals)
+    for idx in np.ndindex(totals.shape):
+        bp[idx], bc[idx], br[idx] = zo.split_budget(int(totals[idx]))
+    Kp, Vp, Qw = wl.prompt(w, 0)
+    K = max(1, min(args.steps, 256))
+    W = max(3, args.warmup)
+    dt, n_sampled, threads = oracle_sample(w, Kp, Vp, Qw, bp, bc, br, W + K)
+    n_units = w.n_layers * w.batch * w.n_kv_heads
+    step_s = dt * n_units / n_sampled
+    sample = "%d of %d units (layer 0) per step, scaled by units; %d steps" % (n_sampled, n_units, K)
+    value = w.batch / step_s
+    print(json.dumps({
+        "impl": "reference", "metric": "decode tokens/s with ZSMerge cache update", "value": value,
+        "unit": "tokens/s", "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": step_s * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch,
+                   "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                   "prompt_len": w.prompt_len, "slots_per_head": int(totals.mean())},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+if __name__ == "__main__":
+    _pre = argparse.ArgumentParser(add_help=False)
+    _pre.add_argument("--impl", default="zsm")
+    if _pre.parse_known_args()[0].impl == "reference":
+        main_reference()
+    else:
+        main()

@@ -1,0 +1,161 @@
+"""GPU parity at the full sizes of workloads c3, c4 (5/10/20 %) and c5, in the launch shape
+the benchmark times (one fused launch over all layers per step).
+
+The whole workload runs on the GPU: prompt pass for every layer, then every decode step
+for every unit.  The oracle cannot redo all of it in test time, so a seeded sample of units
+is recomputed in full -- their prompt pass and every one of their decode steps -- and
+compared element by element; the remaining units are covered by properties that hold at
+any size (occupancy, position bookkeeping, device status).  Inputs are drawn on the GPU by
+the shared seeded recipe; the sampled units' inputs are copied to the host for the oracle.
+"""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from harness import (GpuCache, ParityStats, f64, oracle_step_check, prefill_check, split_budgets,
+                     state_check)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def zb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2503_10714_b200 import binding
+    return binding
+
+
+def run_full_size(zb, oracle, w, n_sample, steps, seed=0):
+    dev = "cuda"
+    totals = wl.head_budgets(w)
+    bp, bc, br = split_budgets(zb, totals)
+    cache = GpuCache(zb, w, bp, bc, br)
+    stats = ParityStats()
+    rs = np.random.RandomState(1000 + seed)
+    sample = {(0, 0, 0), (w.n_layers - 1, w.batch - 1, w.n_kv_heads - 1)}
+    if w.budget is None:  # ragged budgets: make sure the largest and smallest heads are in
+        lo = np.unravel_index(np.argmin(totals), totals.shape)
+        hi = np.unravel_index(np.argmax(totals), totals.shape)
+        sample |= {(int(lo[0]), 0, int(lo[1])), (int(hi[0]), w.batch - 1, int(hi[1]))}
+    while len(sample) < n_sample:
+        sample.add((int(rs.randint(w.n_layers)), int(rs.randint(w.batch)), int(rs.randint(w.n_kv_heads))))
+    sample = sorted(sample)
+    G = w.group
+    try:
+        u = wl.directions(w, dev)
+        units = {}
+        for layer in range(w.n_layers):
+            here = [s for s in sample if s[0] == layer]
+            K, V, Qw = wl.prompt(w, layer, dev, u)
+            dbg = cache.prefill(layer, K, V, Qw, dbg=bool(here))
+            for (l, b, h) in here:
+                small = {k: v[b:b + 1, h:h + 1] for k, v in dbg.items()}
+                units[(l, b, h)] = _prefill_check_one(oracle, cache, l, b, h, K, V, Qw, small, stats, G)
+            del K, V, Qw, dbg
+        assert cache.status() == 0, "device status after the prompt pass"
+
+        ns = len(sample)
+        li = torch.tensor([s[0] for s in sample], device=dev)
+        bi = torch.tensor([s[1] for s in sample], device=dev)
+        hi_ = torch.tensor([s[2] for s in sample], device=dev)
+        q_rec = torch.empty(steps, ns, G, w.head_dim, dtype=w.torch_dtype, device=dev)
+        k_rec = torch.empty(steps, ns, w.head_dim, dtype=w.torch_dtype, device=dev)
+        v_rec = torch.empty_like(k_rec)
+        o_rec = torch.empty_like(q_rec)
+        vic_rec = torch.empty(steps, ns, dtype=torch.int32, device=dev)
+        slot_rec = torch.empty_like(vic_rec)
+        vic_all_min = torch.zeros((), dtype=torch.int32, device=dev)
+        for step in range(steps):
+            q, k, v = wl.decode_inputs(w, step, dev, u)
+            out, vic, slot = cache.decode(q, k, v, layer=-1)
+            qv = q.view(w.n_layers, w.batch, w.n_kv_heads, G, w.head_dim)
+            ov = out.view(w.n_layers, w.batch, w.n_kv_heads, G, w.head_dim)
+            q_rec[step], o_rec[step] = qv[li, bi, hi_], ov[li, bi, hi_]
+            k_rec[step], v_rec[step] = k[li, bi, hi_], v[li, bi, hi_]
+            vic_rec[step], slot_rec[step] = vic[li, bi, hi_], slot[li, bi, hi_]
+            # every unit of a full cache evicts exactly one position per step
+            vic_all_min = torch.minimum(vic_all_min, vic.min())
+        assert cache.status() == 0, "device status after decoding"
+        if (totals < w.prompt_len).all():
+            assert int(vic_all_min.item()) >= 0, "a full unit skipped its eviction"
+
+        q64, k64, v64, o64 = f64(q_rec), f64(k_rec), f64(v_rec), f64(o_rec)
+        vic_h, slot_h = vic_rec.cpu().numpy(), slot_rec.cpu().numpy()
+        for i, key in enumerate(sample):
+            unit = units[key]
+            for step in range(steps):
+                oracle_step_check(unit, q64[step, i], k64[step, i], v64[step, i], o64[step, i],
+                                  vic_h[step, i], slot_h[step, i], w.dtype, stats,
+                                  tag=f"{w.name} step {step} unit {key}")
+            state_check(unit, cache.export(*key), stats, tag=f"{w.name} end state unit {key}")
+
+        # properties for units outside the sample
+        for _ in range(8):
+            l, b, h = int(rs.randint(w.n_layers)), int(rs.randint(w.batch)), int(rs.randint(w.n_kv_heads))
+            st = cache.export(l, b, h)
+            cap = int(bp[l, h] + bc[l, h])
+            assert st["T"] == w.prompt_len + steps
+            assert st["n_live"] == min(cap, w.prompt_len + steps) and st["n_res"] <= br[l, h]
+            pos = np.sort(st["pos"])
+            assert len(np.unique(pos)) == len(pos)
+            n_p = int(bp[l, h])
+            if n_p:
+                np.testing.assert_array_equal(pos[-n_p:], np.arange(st["T"] - n_p, st["T"]))
+            if br[l, h] > 0 and st["n_res"] == br[l, h]:
+                assert st["n_live"] + int(st["w"].sum()) == st["T"]
+    finally:
+        cache.close()
+    assert stats.exact_tie_breaches == 0
+    print(w.name, stats)
+    return stats
+
+
+def _prefill_check_one(oracle, cache, l, b, h, K, V, Qw, dbg_small, stats, G):
+    """prefill_check on host copies of one unit's prompt (keeps host memory small)."""
+    Kh = K[b:b + 1, h:h + 1].cpu()
+    Vh = V[b:b + 1, h:h + 1].cpu()
+    Qh = Qw[b:b + 1, h * G:(h + 1) * G].cpu()
+    return prefill_check(oracle, _Shift(cache, b, h), l, 0, 0, Kh, Vh, Qh, dbg_small, stats,
+                         tag=f"prompt pass unit {(l, b, h)}")
+
+
+class _Shift:
+    """Presents cache unit (layer, b0, h0) under the indices (layer, 0, 0)."""
+
+    def __init__(self, cache, b0, h0):
+        self.c, self.b0, self.h0 = cache, b0, h0
+        self.w = cache.w
+        self.lam, self.alpha = cache.lam, cache.alpha
+        self.bp = cache.bp[:, h0:h0 + 1]
+        self.bc = cache.bc[:, h0:h0 + 1]
+        self.br = cache.br[:, h0:h0 + 1]
+
+    def export(self, layer, b, h):
+        return self.c.export(layer, self.b0 + b, self.h0 + h)
+
+
+def test_c3_llama7b_batch16(zb, oracle):
+    """c3: 32 layers x batch 16 x 32 heads, prompt 16 384, 819 slots per head, 512 steps."""
+    stats = run_full_size(zb, oracle, wl.C3, n_sample=6, steps=wl.C3.decode_steps)
+    assert stats.steps == 6 * 512
+
+
+def test_c4_54k_5pct(zb, oracle):
+    """c4 at 5 %: the benchmark's workload; 54 000-token prompt, 2 700 slots, 1 024 steps."""
+    stats = run_full_size(zb, oracle, wl.C4_5, n_sample=6, steps=wl.C4_5.decode_steps)
+    assert stats.steps == 6 * 1024
+
+
+@pytest.mark.parametrize("w", [wl.C4_10, wl.C4_20], ids=["10pct", "20pct"])
+def test_c4_54k_larger_budgets(zb, oracle, w):
+    """c4 at 10 % and 20 %: 5 400 and 10 800 slots per head (up to 6 score tiles per unit)."""
+    run_full_size(zb, oracle, w, n_sample=3, steps=256)
+
+
+def test_c5_gqa_ragged(zb, oracle):
+    """c5: 8 kv heads shared by 32 query heads, bf16, batch 8, prompt 32 768, per-head budgets
+    drawn in [64, 2048]: the smallest and the largest head are always in the sample."""
+    stats = run_full_size(zb, oracle, wl.C5, n_sample=8, steps=wl.C5.decode_steps)
+    assert stats.steps == 8 * 512
