@@ -194,6 +194,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--cpu-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run a shallower stack than the workload names (profiling captures only; "
+                         "the reported config says so)")
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--consumer-warps", type=int, default=0)
@@ -204,6 +207,8 @@ def main():
     K = max(1, args.steps)
 
     w = w0.replace(seed=w0.seed + 1000 * rank)  # every rank its own sequence
+    if args.layers > 0:
+        w = w.replace(n_layers=args.layers, name=w.name + "_%dlayers" % args.layers)
     from paper_2503_10714_b200 import binding as zb
     totals = wl.head_budgets(w)
     bp = np.zeros_like(totals)
@@ -239,6 +244,7 @@ def main():
             sample_prompt = (Kp.cpu(), Vp.cpu(), Qw.cpu())
         del Kp, Vp, Qw
     del ws
+    torch.cuda.empty_cache()
     if zb.zsm_last_device_status(cache) != 0:
         raise RuntimeError("device status after the prompt pass is not OK")
 
