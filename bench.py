@@ -284,7 +284,7 @@ def main():
     kh = [ks[W + s].cpu().pin_memory() for s in range(Ke)]
     vh = [vs[W + s].cpu().pin_memory() for s in range(Ke)]
     oh = torch.empty_like(qh[0]).pin_memory()
-    for s in range(3):
+    for s in range(min(3, Ke)):
         zb.zsm_decode_step_host(cache, -1, qh[s], kh[s], vh[s], oh, staging)
     torch.cuda.synchronize()
     barrier(world)
