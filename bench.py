@@ -45,14 +45,37 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def recorded_traffic(name):
-    """DRAM bytes per launch from the committed ncu summary of this workload, if any."""
-    path = os.path.join(ROOT, "profiles", "decode_fused_traffic.json")
+KERNEL_SOURCES = ["zsm_decode.cu", "zsm_decode.cuh", "zsm_common.cuh"]
+
+
+def kernel_fingerprint():
+    """sha256 over the decode kernel's sources: ties a recorded ncu figure to the code it came from."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2503_10714_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(w):
+    """DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) for this
+    workload, from profiles/decode_fused_traffic.txt: lines `workload layers bytes fingerprint`
+    taken on a `layers`-deep stack of the workload and scaled here by the units processed
+    (traffic is proportional to units: every unit streams its own slots once).  None when no
+    line matches or the kernel's sources changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "decode_fused_traffic.txt")
+    base = w.name.split("_%dlayers" % w.n_layers)[0]
     try:
+        fp = kernel_fingerprint()
         with open(path) as f:
-            return json.load(f).get(name)
+            for line in f:
+                t = line.split()
+                if len(t) == 4 and not line.startswith("#") and t[0] == base and t[3] == fp:
+                    return int(round(float(t[2]) * w.n_layers / int(t[1])))
     except Exception:
-        return None
+        pass
+    return None
 
 
 class ClockSampler:
@@ -334,7 +357,7 @@ def main():
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_kind,
                      "algorithmic_bytes_per_launch": abytes,
-                     "traffic": recorded_traffic(w.name)},
+                     "traffic": recorded_traffic(w)},
         "prompt_pass": {"ms_total": prefill_ms, "ms_per_layer": prefill_ms / w.n_layers,
                         "window": w.window},
     }

@@ -82,7 +82,7 @@ typedef struct {
     float softmax_scale; /* 0 selects 1/sqrt(head_dim) [Eq. (att_score)] */
     /* Launch tuning of the fused decode kernel; 0 selects the library default. */
     int32_t tune_stages;         /* 16 KiB ring stages per CTA */
-    int32_t tune_ctas_per_sm;    /* persistent CTAs per SM */
+    int32_t tune_ctas_per_sm;    /* persistent CTAs per SM (default 2) */
     int32_t tune_consumer_warps; /* compute warps per CTA (one more warp feeds them) */
 } zsm_config_t;
 

@@ -314,7 +314,9 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
     c->l_stride = (ent_max + 3) & ~3;
 
     // ---- launch plan of the fused decode kernel ----
-    c->ctas_per_sm = cfg->tune_ctas_per_sm > 0 ? cfg->tune_ctas_per_sm : 1;
+    // Two CTAs per SM by default: one CTA's per-unit serial phases (softmax reductions, victim
+    // search, merge) overlap the other's streaming.
+    c->ctas_per_sm = cfg->tune_ctas_per_sm > 0 ? cfg->tune_ctas_per_sm : 2;
     c->consumer_warps = cfg->tune_consumer_warps > 0 ? cfg->tune_consumer_warps : 8;
     if (c->consumer_warps > kMaxConsumerWarps || c->ctas_per_sm > 8) {
         delete c;

@@ -1,6 +1,6 @@
 // Fused decode step of the budgeted KV cache (Algorithm 1 + Eq. (att_score2)).
 //
-// One persistent CTA per SM walks a static list of units.  A producer warp
+// Persistent CTAs (two per SM by default) each walk a static list of units.  A producer warp
 // streams each unit's arrays through a ring of 16 KiB shared-memory stages with
 // 1-D bulk copies (cp.async.bulk + mbarrier); it runs ahead across units, so the
 // tail of one unit (softmax, victim search, merge) overlaps the next unit's loads.
