@@ -135,6 +135,31 @@ zsm_status_t zsm_prefill_compress(zsm_cache_t *c, int32_t layer, const void *K, 
                                   uint8_t *dbg_evicted, int32_t *dbg_targets,
                                   zsm_stream_t stream);
 
+/* zsm_prefill_compress for callers that cannot allocate device memory when they call
+ * (the paper has no counterpart; this is a convenience of the library).  Typical cases: a
+ * serving process whose own memory pool has already reserved the whole GPU, so that a
+ * cudaMalloc made now would fail, or a latency-critical loop that cannot afford the device
+ * synchronisation an allocation may imply.  Arguments, results and status codes are those of
+ * zsm_prefill_compress without `workspace`: the scratch is a fixed array of
+ * ZSM_STATIC_SCRATCH_BYTES that is part of the library image -- every GPU that loads the
+ * library holds those bytes until the process exits -- and the call makes no cudaMalloc,
+ * cudaFree or other allocating call.
+ *   - ZSM_ERR_BUFFER_TOO_SMALL when the prompt needs more scratch than that
+ *     (zsm_prefill_workspace_bytes(c, T, W) tells how much; roughly
+ *     batch*n_kv_heads*T*(13 + 4*G*W) bytes).  Nothing is launched then.
+ *   - The first call on each device looks up the array's device address (with the cache's
+ *     device current, as for every call); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps what the last call left in
+ *     it.  The pass overwrites every entry before it reads it, so nothing needs clearing;
+ *     but two calls whose kernels overlap on the GPU (different streams) race on it.
+ *     Calls on one stream are ordered and safe. */
+#define ZSM_STATIC_SCRATCH_BYTES (16u << 20)
+zsm_status_t zsm_prefill_compress_static(zsm_cache_t *c, int32_t layer, const void *K,
+                                         const void *V, const void *Qw, const float *scores,
+                                         int32_t T, int32_t W, float *dbg_scores,
+                                         uint8_t *dbg_evicted, int32_t *dbg_targets,
+                                         zsm_stream_t stream);
+
 /* One decode step [Algorithm 1 with Eq. (att_score2)], one kernel launch.
  *   layer      0..n_layers-1: that layer's units; tensors have no layer dimension.
  *              -1: every layer in one launch; tensors carry a leading

@@ -30,6 +30,7 @@ DTYPE_CODE = {"f32": ZSM_F32, "f16": ZSM_F16, "bf16": ZSM_BF16,
 # every symbol include/zsm.h declares
 SYMBOLS = ["zsm_split_budget", "zsm_cache_bytes", "zsm_cache_create", "zsm_cache_reset",
            "zsm_cache_free", "zsm_prefill_workspace_bytes", "zsm_prefill_compress",
+           "zsm_prefill_compress_static",
            "zsm_decode_step", "zsm_decode_staging_bytes", "zsm_decode_step_host",
            "zsm_unit_capacity", "zsm_cache_export_unit", "zsm_cache_import_unit",
            "zsm_last_device_status", "zsm_decode_launch_info", "zsm_status_string"]
@@ -66,6 +67,8 @@ _lib.zsm_cache_free.argtypes = [_vp]
 _lib.zsm_prefill_workspace_bytes.argtypes = [_vp, _i32, _i32, C.POINTER(_sz)]
 _lib.zsm_prefill_compress.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp,
                                       _vp, _vp, _vp]
+_lib.zsm_prefill_compress_static.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp,
+                                             _vp, _vp]
 _lib.zsm_decode_step.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.zsm_decode_staging_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
 _lib.zsm_decode_step_host.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -168,6 +171,21 @@ def zsm_prefill_compress(cache, layer, K, V, Qw, scores, T, W, workspace, dbg_sc
                                      workspace.numel() * workspace.element_size(),
                                      _dev(dbg_scores), _dev(dbg_evicted), _dev(dbg_targets),
                                      _stream(stream)), "zsm_prefill_compress")
+
+
+ZSM_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def zsm_prefill_compress_static(cache, layer, K, V, Qw, scores, T, W, dbg_scores=None,
+                                dbg_evicted=None, dbg_targets=None, stream=None):
+    """zsm_prefill_compress with the library's own fixed scratch array instead of a workspace
+    tensor, for callers that cannot allocate device memory at the time of the call.  Raises
+    ZsmError(ZSM_ERR_BUFFER_TOO_SMALL) when the prompt needs more than
+    ZSM_STATIC_SCRATCH_BYTES; calls on different streams must not overlap."""
+    _check(_lib.zsm_prefill_compress_static(cache, int(layer), _dev(K), _dev(V), _dev(Qw),
+                                            _dev(scores), int(T), int(W), _dev(dbg_scores),
+                                            _dev(dbg_evicted), _dev(dbg_targets),
+                                            _stream(stream)), "zsm_prefill_compress_static")
 
 
 def zsm_decode_step(cache, layer, q, k_new, v_new, out, victim_pos=None, merge_slot=None,
