@@ -162,6 +162,18 @@ def max_over_ranks(x: float, world: int) -> float:
     return float(t.item())
 
 
+def whole_job_throughput(ms_local: float, tokens_per_rank: int, world: int):
+    """Tokens of all ranks divided by the slowest rank's device time (weak scaling: every rank
+    processes its own `tokens_per_rank`).  Returns (tokens/s, max-over-ranks ms)."""
+    ms_total = max_over_ranks(ms_local, world)
+    return world * tokens_per_rank / (ms_total * 1e-3), ms_total
+
+
+def rank_workload(w0, rank: int):
+    """Each rank decodes its own sequence: same shape, its own seed.  No data-path collective."""
+    return w0.replace(seed=w0.seed + 1000 * rank)
+
+
 def barrier(world):
     if world > 1:
         import torch.distributed as dist
@@ -229,7 +241,7 @@ def main():
     W = max(3, args.warmup)
     K = max(1, args.steps)
 
-    w = w0.replace(seed=w0.seed + 1000 * rank)  # every rank its own sequence
+    w = rank_workload(w0, rank)
     if args.layers > 0:
         w = w.replace(n_layers=args.layers, name=w.name + "_%dlayers" % args.layers)
     from paper_2503_10714_b200 import binding as zb
@@ -295,7 +307,7 @@ def main():
     torch.cuda.synchronize()
     barrier(world)
     ms_local = ev0.elapsed_time(ev1)
-    ms_total = max_over_ranks(ms_local, world)
+    value, ms_total = whole_job_throughput(ms_local, w.batch * K, world)
     ms_per_step = ms_total / K
     if zb.zsm_last_device_status(cache) != 0:
         raise RuntimeError("device status after the timed region is not OK")
@@ -333,7 +345,7 @@ def main():
     grid, block, smem = zb.zsm_decode_launch_info(cache, -1)
     line = {
         "metric": "decode tokens/s with ZSMerge cache update",
-        "value": world * w.batch * K / (ms_total * 1e-3),
+        "value": value,
         "unit": "tokens/s",
         "n_gpus": world,
         "steps": K,
