@@ -83,7 +83,8 @@ typedef struct {
     /* Launch tuning of the fused decode kernel; 0 selects the library default. */
     int32_t tune_stages;         /* 16 KiB ring stages per CTA */
     int32_t tune_ctas_per_sm;    /* persistent CTAs per SM (default 2) */
-    int32_t tune_consumer_warps; /* compute warps per CTA (one more warp feeds them) */
+    int32_t tune_consumer_warps; /* compute warps per CTA, at most 8 (two more warps feed them
+                                  * and write the cache update back) */
 } zsm_config_t;
 
 /* Budget split of App. C.2: B_p = floor(tail_ratio*B); B_r = round(dense_ratio*

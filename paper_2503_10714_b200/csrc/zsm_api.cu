@@ -341,7 +341,7 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
         return ZSM_ERR_UNSUPPORTED;
     }
     int occ = 0;
-    int rc = prepare_decode_fused(s.dtype, s.D, s.G, c->smem_bytes, (c->consumer_warps + 1) * 32, &occ);
+    int rc = prepare_decode_fused(s.dtype, s.D, s.G, c->smem_bytes, (c->consumer_warps + kExtraWarps) * 32, &occ);
     if (rc != 0 || prepare_prefill(s.dtype, s.D) != 0) {
         delete c;
         return rc == -1 ? ZSM_ERR_UNSUPPORTED : ZSM_ERR_CUDA;
@@ -419,7 +419,7 @@ zsm_status_t zsm_decode_launch_info(const zsm_cache_t *c, int32_t layer, int32_t
                                     int32_t *block, int32_t *dynamic_smem_bytes) {
     if (!c || layer < -1 || layer >= c->s.L) return ZSM_ERR_INVALID_ARG;
     if (grid) *grid = layer < 0 ? c->grid_all : c->grid_layer;
-    if (block) *block = (c->consumer_warps + 1) * 32;
+    if (block) *block = (c->consumer_warps + kExtraWarps) * 32;
     if (dynamic_smem_bytes) *dynamic_smem_bytes = c->smem_bytes;
     return ZSM_OK;
 }

@@ -1,32 +1,53 @@
 // Fused decode step of the budgeted KV cache (Algorithm 1 + Eq. (att_score2)).
 //
-// Persistent CTAs (two per SM by default) each walk a static list of units.  A producer warp
-// streams each unit's arrays through a ring of 16 KiB shared-memory stages with
-// 1-D bulk copies (cp.async.bulk + mbarrier); it runs ahead across units, so the
-// tail of one unit (softmax, victim search, merge) overlaps the next unit's loads.
-// Consumer warps take the tiles in order:
+// Persistent CTAs (two per SM by default) each walk a static list of units.  Three roles:
 //
+// Producer warp: streams each unit's arrays through a ring of 16 KiB shared-memory stages
+// with 1-D bulk copies (cp.async.bulk + mbarrier); it runs ahead across units, so a unit's
+// serial phases (softmax reductions, victim search) overlap the next unit's loads.
+//
+// Consumer warps take the tiles in order:
 //   header   counters, q (G heads), k_new, v_new, fusion counts w
 //   K tiles  logits q.k/sqrt(d) of every live token slot          (D1)
 //   Kr tiles logits of the merged slots, + alpha*ln w             (D1, Eq. (att_score2))
 //   -- softmax over slots + new token                             (D2)
 //   meta     score, pos: s <- lambda*s + mean_g a_hat; running argmin of
 //            (s, pos) over slots that left the proximity window   (D4, D5)
-//   -- residual target: fill, or argmax_r k_r.k_victim and the incremental mean (D6)
+//   -- the victim goes to the tail warp through a mailbox
 //   V tiles, Vr tiles   o = sum a_hat v                            (D3)
-//   -- write o; new token into the victim's slot; merged rows; counters (D6, D7)
+//   -- write o
 //
-// K and V rows cross HBM exactly once per step; grouped query heads share them.
+// Tail warp: off the streaming path, per unit: residual target (free slot, or argmax_r
+// k_r.k_victim and the incremental mean; D6), then -- once the unit's last tile has been
+// read -- the new token into the victim's slot, the merged rows, counts and counters (D6, D7).
+//
+// K and V rows cross HBM exactly once per step; grouped query heads share them.  Weights are
+// kept interleaved, [slot][g], so one shared-memory load serves all heads of a group.
 #include "zsm_decode.cuh"
 
 namespace zsm {
 
 namespace {
 
-constexpr int kMaxThreads = (kMaxConsumerWarps + 1) * 32;
+constexpr int kMaxThreads = (kMaxConsumerWarps + kExtraWarps) * 32;
 
 // "where" codes recorded with a timeout
-enum : int32_t { W_PRODUCER = 1, W_HEADER = 2, W_K = 3, W_KR = 4, W_META = 5, W_V = 6, W_VR = 7 };
+enum : int32_t {
+    W_PRODUCER = 1, W_HEADER = 2, W_K = 3, W_KR = 4, W_META = 5, W_V = 6, W_VR = 7,
+    W_MAIL_FREE = 8, W_TAIL_POST = 9, W_TAIL_VDONE = 10
+};
+
+// Fixed part of a mailbox (kMailFixed bytes), followed by k_new, v_new (storage dtype) and w.
+struct __align__(16) Mail {
+    int4 cnt;
+    UnitDesc d;
+    int32_t victim_slot;  // >= 0 token slot; -2 the new token itself (B_p = 0); -1 none
+    int32_t victim_pos;
+    int32_t evict;
+    float s_tok;
+    int32_t pad[4];
+};
+static_assert(sizeof(Mail) == kMailFixed, "mailbox header size");
 
 template <int LANES>
 __device__ __forceinline__ float group_sum(float v) {
@@ -35,10 +56,103 @@ __device__ __forceinline__ float group_sum(float v) {
     return v;
 }
 
+__host__ __device__ constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
+
+// Sums each of the N values over the LG lanes of a group with a transposing butterfly: while
+// more than one value is left, a step halves the values a lane carries instead of repeating
+// the exchange for each.  Afterwards v[0 .. max(1, N/LG)) hold complete sums of the values
+// treduce_index(l) + i.  N and LG are powers of two; l is the lane's index in its group.
+template <int N, int LG>
+__device__ __forceinline__ void treduce(float (&v)[N], int l) {
+    constexpr int STEPS = ilog2(LG);
+#pragma unroll
+    for (int s = 0; s < STEPS; ++s) {
+        const int off = LG >> (s + 1);
+        const int n = (N >> s) > 1 ? (N >> s) : 1;
+        if (n > 1) {
+            const bool up = (l & off) != 0;
+#pragma unroll
+            for (int i = 0; i < n / 2; ++i) {
+                const float keep = up ? v[i + n / 2] : v[i];
+                const float send = up ? v[i] : v[i + n / 2];
+                v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            }
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
+        }
+    }
+}
+
+template <int N, int LG>
+__device__ __forceinline__ int treduce_index(int l) {
+    constexpr int STEPS = ilog2(LG);
+    int idx = 0;
+#pragma unroll
+    for (int s = 0; s < STEPS; ++s) {
+        const int off = LG >> (s + 1);
+        const int n = (N >> s) > 1 ? (N >> s) : 1;
+        if (n > 1 && (l & off)) idx += n / 2;
+    }
+    return idx;
+}
+
+// G consecutive floats (one slot's weights for the whole group).
+template <int G>
+__device__ __forceinline__ void load_group(const float *p, float (&v)[G]) {
+    if constexpr (G == 1) {
+        v[0] = p[0];
+    } else if constexpr (G == 2) {
+        const float2 t = *reinterpret_cast<const float2 *>(p);
+        v[0] = t.x;
+        v[1] = t.y;
+    } else {
+#pragma unroll
+        for (int i = 0; i < G / 4; ++i) {
+            const float4 t = reinterpret_cast<const float4 *>(p)[i];
+            v[4 * i] = t.x;
+            v[4 * i + 1] = t.y;
+            v[4 * i + 2] = t.z;
+            v[4 * i + 3] = t.w;
+        }
+    }
+}
+
+template <int G>
+__device__ __forceinline__ void store_group(float *p, const float (&v)[G]) {
+    if constexpr (G == 1) {
+        p[0] = v[0];
+    } else if constexpr (G == 2) {
+        *reinterpret_cast<float2 *>(p) = make_float2(v[0], v[1]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < G / 4; ++i)
+            reinterpret_cast<float4 *>(p)[i] =
+                make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    }
+}
+
+// Four consecutive elements of a row in the storage dtype, widened.
+template <typename T>
+__device__ __forceinline__ void load4(const T *p, float (&f)[4]) {
+    if constexpr (sizeof(T) == 4) {
+        const float4 t = *reinterpret_cast<const float4 *>(p);
+        f[0] = t.x;
+        f[1] = t.y;
+        f[2] = t.z;
+        f[3] = t.w;
+    } else {
+        const uint2 t = *reinterpret_cast<const uint2 *>(p);
+        const T *e = reinterpret_cast<const T *>(&t);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) f[i] = Elem<T>::to_float(e[i]);
+    }
+}
+
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const DecodeParams p) {
     using E = Elem<T>;
     constexpr int EPL = E::EPL;               // elements per 16-byte lane load
+    constexpr int EP2 = EPL / 2;
     constexpr int ROWB = D * (int)sizeof(T);  // bytes per token row
     constexpr int LPR = D / EPL;              // lanes per token row
     constexpr int RPW = 32 / LPR;             // token rows per warp-wide load
@@ -53,10 +167,13 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
     constexpr int HDR_K = HDR_Q + G * ROWB;
     constexpr int HDR_V = HDR_K + ROWB;
     constexpr int HDR_W = HDR_V + ROWB;
-    constexpr int UB = 4;                     // row groups in flight per warp
+    constexpr int UBK = G <= 2 ? 4 : 2;       // row groups in flight per warp, logits pass
+    constexpr int UBV = G <= 4 ? 4 : 2;       // same, output pass
+    constexpr int NV = G * UBK;               // partial dot products a lane carries
+    constexpr int NF = NV > LPR ? NV / LPR : 1;
 
     extern __shared__ __align__(128) uint8_t smem[];
-    const int NW = (blockDim.x >> 5) - 1;  // consumer warps
+    const int NW = (blockDim.x >> 5) - kExtraWarps;  // consumer warps
     const int NT = NW * 32;
     const int S = p.stages;
     const int LS = p.l_stride;
@@ -65,22 +182,16 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
     uint8_t *ring = smem + L.ring;
     uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + L.bars);
     uint64_t *empty_bar = full_bar + S;
-    volatile int32_t *flags = reinterpret_cast<volatile int32_t *>(smem + L.flags);
-    volatile int32_t *abort_flag = flags;  // flags[0]
-    float *probs = reinterpret_cast<float *>(smem + L.probs);
+    uint64_t *post_bar = empty_bar + S;   // [2] consumers -> tail: the unit's victim is known
+    uint64_t *vdone_bar = post_bar + 2;   // [2] consumers -> tail: the unit's last tile was read
+    uint64_t *freed_bar = vdone_bar + 2;  // [2] tail -> consumers: the mailbox may be reused
+    volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(smem + L.flags);
+    float *probs = reinterpret_cast<float *>(smem + L.probs);  // [slot][G]
     float *qf = reinterpret_cast<float *>(smem + L.qf);
-    uint4 *kn_raw = reinterpret_cast<uint4 *>(smem + L.kn);
-    uint4 *vn_raw = reinterpret_cast<uint4 *>(smem + L.vn);
-    uint32_t *w_s = reinterpret_cast<uint32_t *>(smem + L.w);
     float *opart = reinterpret_cast<float *>(smem + L.opart);
     float *redf = reinterpret_cast<float *>(smem + L.redf);
     float *redf2 = redf + kMaxConsumerWarps * 8;
     uint64_t *red64 = reinterpret_cast<uint64_t *>(smem + L.red64);
-    float *dots = reinterpret_cast<float *>(smem + L.dots);
-    float *kc = reinterpret_cast<float *>(smem + L.rows);
-    float *vc = kc + D;
-    float *mk = vc + D;
-    float *mv = mk + D;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -91,7 +202,12 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], NW);
         }
-        flags[0] = 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&post_bar[b], 1);
+            mbar_init(&vdone_bar[b], 1);
+            mbar_init(&freed_bar[b], 1);
+        }
+        *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -211,13 +327,158 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
         return;
     }
 
+    const int l32 = lane % LPR32;  // 16-byte column of an fp32 residual row
+    const int sub32 = lane / LPR32;
+
+    // =====================================================================
+    // Tail warp: residual fill / merge and the write-back of each unit.
+    // =====================================================================
+    if (warp == NW + 1) {
+        for (int n = 0; n < last - first; ++n) {
+            const int mb = n & 1;
+            const uint32_t mph = (n >> 1) & 1u;
+            const uint8_t *mailp = smem + L.mail + mb * L.mail_stride;
+            if (!mbar_wait_bounded(&post_bar[mb], mph, abort_flag, p.status, W_TAIL_POST)) return;
+            const Mail *m = reinterpret_cast<const Mail *>(mailp);
+            const uint4 *kn_raw = reinterpret_cast<const uint4 *>(mailp + kMailFixed);
+            const uint4 *vn_raw = reinterpret_cast<const uint4 *>(mailp + kMailFixed + ROWB);
+            const uint32_t *w_s = reinterpret_cast<const uint32_t *>(mailp + kMailFixed + 2 * ROWB);
+            const int4 cnt = m->cnt;
+            const UnitDesc d = m->d;
+            const int cap = d.Bp + d.Bc;
+            const int n_live = min(max(cnt.x, 0), cap);
+            const int n_res = min(max(cnt.y, 0), d.Br);
+            const int Tpos = cnt.z;
+            const int ul = d.unit - p.unit_base;
+            const int victim_slot = m->victim_slot;
+            const int victim_pos = m->victim_pos;
+            const bool evict = m->evict != 0;
+            const float s_tok = m->s_tok;
+            const bool have_victim = evict && victim_slot != -1;
+
+            int merge_slot = -1;  // report: slot merged into, -2 fill, -1 none
+            int res_target = -1;  // residual row to write
+            uint32_t res_w = 0;
+            float mk[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+            float *Kr_g = reinterpret_cast<float *>(p.base + d.kr_off);
+            float *Vr_g = reinterpret_cast<float *>(p.base + d.vr_off);
+            if (have_victim && d.Br > 0) {
+                float kc[4], vc[4];
+                if (victim_slot >= 0) {
+                    load4<T>(reinterpret_cast<const T *>(p.base + d.k_off + (size_t)victim_slot * ROWB) + l32 * 4, kc);
+                    load4<T>(reinterpret_cast<const T *>(p.base + d.v_off + (size_t)victim_slot * ROWB) + l32 * 4, vc);
+                } else {
+                    load4<T>(reinterpret_cast<const T *>(kn_raw) + l32 * 4, kc);
+                    load4<T>(reinterpret_cast<const T *>(vn_raw) + l32 * 4, vc);
+                }
+                if (n_res < d.Br) {
+                    // Alg. 1: a free residual slot takes the token as it is
+                    res_target = n_res;
+                    res_w = 1;
+                    merge_slot = -2;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        mk[e] = kc[e];
+                        mv[e] = vc[e];
+                    }
+                } else {
+                    // Eq. (hatr): raw dot product with every merged key; ties to the lowest slot
+                    float bd = -INFINITY;
+                    int br = 0x7fffffff;
+                    for (int r0 = 0; r0 < n_res; r0 += 4 * RPW32) {
+                        float4 kr[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int r = r0 + u * RPW32 + sub32;
+                            kr[u] = r < n_res ? *reinterpret_cast<const float4 *>(Kr_g + (size_t)r * D + l32 * 4)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int r = r0 + u * RPW32 + sub32;
+                            float acc = 0.f;
+                            acc = fmaf(kr[u].x, kc[0], acc);
+                            acc = fmaf(kr[u].y, kc[1], acc);
+                            acc = fmaf(kr[u].z, kc[2], acc);
+                            acc = fmaf(kr[u].w, kc[3], acc);
+                            acc = group_sum<LPR32>(acc);
+                            if (r < n_res && (br == 0x7fffffff || acc > bd)) {
+                                bd = acc;
+                                br = r;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int off = LPR32; off < 32; off <<= 1) {
+                        const float od = __shfl_xor_sync(0xffffffffu, bd, off);
+                        const int orr = __shfl_xor_sync(0xffffffffu, br, off);
+                        if (orr != 0x7fffffff && (br == 0x7fffffff || od > bd || (od == bd && orr < br))) {
+                            bd = od;
+                            br = orr;
+                        }
+                    }
+                    res_target = br;
+                    merge_slot = br;
+                    const uint32_t wr_u = w_s[br];
+                    res_w = wr_u + 1u;
+                    const float wr = static_cast<float>(wr_u);
+                    // Eq. (kvr): incremental mean of key and value
+                    const float4 ko = *reinterpret_cast<const float4 *>(Kr_g + (size_t)br * D + l32 * 4);
+                    const float4 vo = *reinterpret_cast<const float4 *>(Vr_g + (size_t)br * D + l32 * 4);
+                    const float kof[4] = {ko.x, ko.y, ko.z, ko.w}, vof[4] = {vo.x, vo.y, vo.z, vo.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        mk[e] = fmaf(wr, kof[e], kc[e]) / (wr + 1.0f);
+                        mv[e] = fmaf(wr, vof[e], vc[e]) / (wr + 1.0f);
+                    }
+                }
+            }
+
+            // every tile of this unit has been read: its rows may now be overwritten
+            if (!mbar_wait_bounded(&vdone_bar[mb], mph, abort_flag, p.status, W_TAIL_VDONE)) return;
+            const bool insert = evict ? (have_victim && victim_slot >= 0) : true;
+            const int ins_slot = evict ? victim_slot : n_live;
+            if (insert) {
+                uint4 *kd = reinterpret_cast<uint4 *>(p.base + d.k_off + (size_t)ins_slot * ROWB);
+                uint4 *vd = reinterpret_cast<uint4 *>(p.base + d.v_off + (size_t)ins_slot * ROWB);
+                for (int c = lane; c < ROWB / 16; c += 32) {
+                    kd[c] = kn_raw[c];
+                    vd[c] = vn_raw[c];
+                }
+            }
+            if (res_target >= 0 && sub32 == 0) {
+                *reinterpret_cast<float4 *>(Kr_g + (size_t)res_target * D + l32 * 4) =
+                    make_float4(mk[0], mk[1], mk[2], mk[3]);
+                *reinterpret_cast<float4 *>(Vr_g + (size_t)res_target * D + l32 * 4) =
+                    make_float4(mv[0], mv[1], mv[2], mv[3]);
+            }
+            if (lane == 0) {
+                if (insert) {
+                    reinterpret_cast<float *>(p.base + d.score_off)[ins_slot] = s_tok;
+                    reinterpret_cast<int32_t *>(p.base + d.pos_off)[ins_slot] = Tpos;
+                }
+                if (res_target >= 0)
+                    reinterpret_cast<uint32_t *>(p.base + d.w_off)[res_target] = res_w;
+                UnitCounters c;
+                c.n_live = n_live + ((!evict) ? 1 : 0);
+                c.n_res = n_res + ((merge_slot == -2) ? 1 : 0);
+                c.T = Tpos + 1;
+                c.pad = 0;
+                *reinterpret_cast<int4 *>(p.counters + d.unit) = *reinterpret_cast<int4 *>(&c);
+                if (p.victim_pos) p.victim_pos[ul] = victim_pos;
+                if (p.merge_slot) p.merge_slot[ul] = merge_slot;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&freed_bar[mb]);
+        }
+        return;
+    }
+
     // =====================================================================
     // Consumers
     // =====================================================================
-    const int l = lane % LPR;      // 16-byte column of a token row
-    const int sub = lane / LPR;    // which of the RPW rows of a warp-wide load
-    const int l32 = lane % LPR32;  // same for fp32 residual rows
-    const int sub32 = lane / LPR32;
+    const int l = lane % LPR;    // 16-byte column of a token row
+    const int sub = lane / LPR;  // which of the RPW rows of a warp-wide load
 
     int cs = 0;
     uint32_t cph = 0;
@@ -235,10 +496,25 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
     };
     auto csync = [&]() { named_bar_sync(1, NT); };
 
+    // where this lane's sums land after the transposing reduction of the logits pass
+    const int tr_idx = treduce_index<NV, LPR>(l);
+    const bool tr_writer = (NV >= LPR) || ((l & (LPR / (NV < LPR ? NV : LPR) - 1)) == 0);
+
     for (int i = first; i < last; ++i) {
+        const int n = i - first;
+        const int mb = n & 1;
+        const uint32_t mph = (n >> 1) & 1u;
+        uint8_t *mailp = smem + L.mail + mb * L.mail_stride;
+        Mail *mail = reinterpret_cast<Mail *>(mailp);
+        uint4 *kn_raw = reinterpret_cast<uint4 *>(mailp + kMailFixed);
+        uint4 *vn_raw = reinterpret_cast<uint4 *>(mailp + kMailFixed + ROWB);
+        uint32_t *w_s = reinterpret_cast<uint32_t *>(mailp + kMailFixed + 2 * ROWB);
+
         // ---------------- header ----------------
         const uint8_t *h = wait_full(W_HEADER);
         if (!h) return;
+        // the tail warp is done with this mailbox's previous unit (two units back)
+        if (!mbar_wait_bounded(&freed_bar[mb], mph ^ 1u, abort_flag, p.status, W_MAIL_FREE)) return;
         const int4 cnt = *reinterpret_cast<const int4 *>(h);
         const UnitDesc d = *reinterpret_cast<const UnitDesc *>(h + HDR_D);
         const int cap = d.Bp + d.Bc;
@@ -251,11 +527,14 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
         const int Tpos = cnt.z;
         const int n_ent = n_live + n_res + 1;
 
-        float qreg[G][EPL];
+        float2 q2[G][EP2];
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             const uint4 raw = *reinterpret_cast<const uint4 *>(h + HDR_Q + g * ROWB + l * 16);
-            E::widen(raw, qreg[g]);
+            float f[EPL];
+            E::widen(raw, f);
+#pragma unroll
+            for (int e = 0; e < EP2; ++e) q2[g][e] = make_float2(f[2 * e], f[2 * e + 1]);
         }
         {
             const T *qs = reinterpret_cast<const T *>(h + HDR_Q);
@@ -268,6 +547,10 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
             }
             const uint32_t *ws = reinterpret_cast<const uint32_t *>(h + HDR_W);
             for (int k = tid; k < br_pad; k += NT) w_s[k] = ws[k];
+            if (tid == 0) {
+                mail->cnt = cnt;
+                mail->d = d;
+            }
         }
         release();
 
@@ -276,33 +559,43 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
             const uint8_t *tile = wait_full(W_K);
             if (!tile) return;
             const int rows = min(R, n_live - r0);
-            for (int base = warp * RPW; base < rows; base += NW * RPW * UB) {
-                uint4 raw[UB];
+            for (int base = warp * RPW; base < rows; base += NW * RPW * UBK) {
+                uint4 raw[UBK];
 #pragma unroll
-                for (int u = 0; u < UB; ++u) {
+                for (int u = 0; u < UBK; ++u) {
                     const int row = base + u * NW * RPW + sub;
                     raw[u] = row < rows
                                  ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
                                  : make_uint4(0, 0, 0, 0);
                 }
+                float v[NV];
 #pragma unroll
-                for (int u = 0; u < UB; ++u) {
-                    const int row = base + u * NW * RPW + sub;
+                for (int u = 0; u < UBK; ++u) {
                     float f[EPL];
                     E::widen(raw[u], f);
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
-                        float acc = 0.f;
+                        float2 a = make_float2(0.f, 0.f);
 #pragma unroll
-                        for (int e = 0; e < EPL; ++e) acc = fmaf(qreg[g][e], f[e], acc);
-                        acc = group_sum<LPR>(acc);
-                        if (l == 0 && row < rows) probs[g * LS + r0 + row] = acc * p.scale;
+                        for (int e = 0; e < EP2; ++e)
+                            a = __ffma2_rn(q2[g][e], make_float2(f[2 * e], f[2 * e + 1]), a);
+                        v[u * G + g] = a.x + a.y;
+                    }
+                }
+                treduce<NV, LPR>(v, l);
+                if (tr_writer) {
+#pragma unroll
+                    for (int k = 0; k < NF; ++k) {
+                        const int id = tr_idx + k;
+                        const int u = id / G, g = id % G;
+                        const int row = base + u * NW * RPW + sub;
+                        if (row < rows) probs[(r0 + row) * G + g] = v[k] * p.scale;
                     }
                 }
             }
             release();
         }
-        csync();  // qf, kn_raw, w_s of this unit are in place
+        csync();  // qf and the mailbox arrays of this unit are in place
 
         // ---------------- D1: logits of the merged slots, + alpha ln w ----------------
         for (int r0 = 0; r0 < n_res; r0 += R32) {
@@ -323,7 +616,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
                     acc = fmaf(qv.w, kr.w, acc);
                     acc = group_sum<LPR32>(acc);
                     if (l32 == 0 && row < rows)
-                        probs[g * LS + n_live + r0 + row] =
+                        probs[(n_live + r0 + row) * G + g] =
                             fmaf(p.alpha, logf(static_cast<float>(w_s[r0 + row])), acc * p.scale);
                 }
             }
@@ -340,7 +633,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
 #pragma unroll
                 for (int e = 0; e < EPL; ++e) acc = fmaf(qg[e], f[e], acc);
                 acc = group_sum<32>(acc);
-                if (lane == 0) probs[g * LS + n_ent - 1] = acc * p.scale;
+                if (lane == 0) probs[(n_ent - 1) * G + g] = acc * p.scale;
             }
         }
         csync();
@@ -350,8 +643,10 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
 #pragma unroll
         for (int g = 0; g < G; ++g) mx[g] = -INFINITY;
         for (int j = tid; j < n_ent; j += NT) {
+            float pv[G];
+            load_group<G>(probs + j * G, pv);
 #pragma unroll
-            for (int g = 0; g < G; ++g) mx[g] = fmaxf(mx[g], probs[g * LS + j]);
+            for (int g = 0; g < G; ++g) mx[g] = fmaxf(mx[g], pv[g]);
         }
 #pragma unroll
         for (int g = 0; g < G; ++g) {
@@ -372,12 +667,14 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
 #pragma unroll
             for (int g = 0; g < G; ++g) sm[g] = 0.f;
             for (int j = tid; j < n_ent; j += NT) {
+                float pv[G];
+                load_group<G>(probs + j * G, pv);
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    const float e = expf(probs[g * LS + j] - mx[g]);
-                    probs[g * LS + j] = e;
-                    sm[g] += e;
+                    pv[g] = expf(pv[g] - mx[g]);
+                    sm[g] += pv[g];
                 }
+                store_group<G>(probs + j * G, pv);
             }
 #pragma unroll
             for (int g = 0; g < G; ++g) {
@@ -394,22 +691,23 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
         }
 
         // ---------------- D4 + D5: score update and victim search ----------------
-        const bool evict = (n_live == cap);  // the new token does not fit: Alg. 1 l.7-11
+        const bool evict = (n_live == cap);  // the new token does not fit: Alg. 1, overflow branch
         const int cut = Tpos - d.Bp;         // positions <= cut have left the proximity window
         float *score_g = reinterpret_cast<float *>(p.base + d.score_off);
-        int32_t *pos_g = reinterpret_cast<int32_t *>(p.base + d.pos_off);
         uint64_t best = ~0ull;
         int best_slot = -1;
         for (int j0 = 0; j0 < n_live; j0 += RM) {
             const uint8_t *tile = wait_full(W_META);
             if (!tile) return;
-            const int n = min(RM, n_live - j0);
+            const int nn = min(RM, n_live - j0);
             const float *ts = reinterpret_cast<const float *>(tile);
             const int32_t *tp = reinterpret_cast<const int32_t *>(tile + RM * 4);
-            for (int k = tid; k < n; k += NT) {
+            for (int k = tid; k < nn; k += NT) {
+                float pv[G];
+                load_group<G>(probs + (j0 + k) * G, pv);
                 float a = 0.f;
 #pragma unroll
-                for (int g = 0; g < G; ++g) a += probs[g * LS + j0 + k] * inv[g];
+                for (int g = 0; g < G; ++g) a += pv[g] * inv[g];
                 a *= (1.0f / G);
                 const float s_new = fmaf(p.lambda, ts[k], a);  // Eq. (score)
                 score_g[j0 + k] = s_new;
@@ -427,11 +725,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
         }
         float s_tok = 0.f;  // first score of the new token: its own attention weight
 #pragma unroll
-        for (int g = 0; g < G; ++g) s_tok += probs[g * LS + n_ent - 1] * inv[g];
+        for (int g = 0; g < G; ++g) s_tok += probs[(n_ent - 1) * G + g] * inv[g];
         s_tok *= (1.0f / G);
 
-        int victim_slot = -1;  // >= 0: token slot; -2: the new token itself (B_p = 0)
-        int victim_pos = -1;
         if (evict) {
             if (tid == 0 && d.Bp == 0) {
                 const uint64_t key =
@@ -455,144 +751,74 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
                 red64[warp * 2 + 1] = static_cast<uint64_t>(static_cast<uint32_t>(best_slot));
             }
             csync();
-            best = red64[0];
-            best_slot = static_cast<int>(static_cast<uint32_t>(red64[1]));
-            for (int wv = 1; wv < NW; ++wv) {
-                const uint64_t ob = red64[wv * 2];
-                if (ob < best) {
-                    best = ob;
-                    best_slot = static_cast<int>(static_cast<uint32_t>(red64[wv * 2 + 1]));
-                }
-            }
-            if (best == ~0ull) {
-                if (tid == 0) dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 2);
-            } else {
-                victim_slot = best_slot;
-                victim_pos = static_cast<int>(static_cast<uint32_t>(best & 0xffffffffull));
-            }
         }
-        const bool have_victim = evict && victim_slot != -1;
-
-        // ---------------- D6: where the victim goes ----------------
-        int merge_slot = -1;  // report: slot merged into, -2 fill, -1 none
-        int res_target = -1;  // residual row to write after the V pass
-        uint32_t res_w = 0;
-        if (have_victim && d.Br > 0) {
-            if (warp == 0) {
-                for (int k = lane; k < LPR; k += 32) {
-                    float f[EPL];
-                    const uint4 raw = victim_slot >= 0
-                                          ? *reinterpret_cast<const uint4 *>(
-                                                p.base + d.k_off + (size_t)victim_slot * ROWB + k * 16)
-                                          : kn_raw[k];
-                    E::widen(raw, f);
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) kc[k * EPL + e] = f[e];
+        // Thread 0 settles the victim and hands the unit's update to the tail warp.  Every
+        // store the consumer warps made for this unit so far (mailbox arrays, updated scores)
+        // is ordered before the hand-over by the barriers above.
+        if (tid == 0) {
+            int victim_slot = -1;  // >= 0: token slot; -2: the new token itself (B_p = 0)
+            int victim_pos = -1;
+            if (evict) {
+                best = red64[0];
+                best_slot = static_cast<int>(static_cast<uint32_t>(red64[1]));
+                for (int wv = 1; wv < NW; ++wv) {
+                    const uint64_t ob = red64[wv * 2];
+                    if (ob < best) {
+                        best = ob;
+                        best_slot = static_cast<int>(static_cast<uint32_t>(red64[wv * 2 + 1]));
+                    }
+                }
+                if (best == ~0ull) {
+                    dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 2);
+                } else {
+                    victim_slot = best_slot;
+                    victim_pos = static_cast<int>(static_cast<uint32_t>(best & 0xffffffffull));
                 }
             }
-            if (warp == (NW > 1 ? 1 : 0)) {
-                for (int k = lane; k < LPR; k += 32) {
-                    float f[EPL];
-                    const uint4 raw = victim_slot >= 0
-                                          ? *reinterpret_cast<const uint4 *>(
-                                                p.base + d.v_off + (size_t)victim_slot * ROWB + k * 16)
-                                          : vn_raw[k];
-                    E::widen(raw, f);
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) vc[k * EPL + e] = f[e];
-                }
-            }
-            csync();
-            const float *Kr_g = reinterpret_cast<const float *>(p.base + d.kr_off);
-            const float *Vr_g = reinterpret_cast<const float *>(p.base + d.vr_off);
-            if (n_res < d.Br) {
-                // Alg. 1 l.12-13: a free residual slot takes the token as it is
-                res_target = n_res;
-                res_w = 1;
-                merge_slot = -2;
-                for (int k = tid; k < D; k += NT) {
-                    mk[k] = kc[k];
-                    mv[k] = vc[k];
-                }
-            } else {
-                // Eq. (hatr): raw dot product with every merged key
-                for (int r = warp; r < n_res; r += NW) {
-                    float acc = 0.f;
-                    for (int k = lane; k < LPR32; k += 32) {
-                        const float4 kr = *reinterpret_cast<const float4 *>(Kr_g + (size_t)r * D + k * 4);
-                        acc = fmaf(kr.x, kc[k * 4 + 0], acc);
-                        acc = fmaf(kr.y, kc[k * 4 + 1], acc);
-                        acc = fmaf(kr.z, kc[k * 4 + 2], acc);
-                        acc = fmaf(kr.w, kc[k * 4 + 3], acc);
-                    }
-                    acc = group_sum<32>(acc);
-                    if (lane == 0) dots[r] = acc;
-                }
-                csync();
-                if (warp == 0) {
-                    float bd = -INFINITY;
-                    int br = 0x7fffffff;
-                    for (int r = lane; r < n_res; r += 32) {
-                        const float dv = dots[r];
-                        if (br == 0x7fffffff || dv > bd) {
-                            bd = dv;
-                            br = r;
-                        }
-                    }
-#pragma unroll
-                    for (int off = 16; off >= 1; off >>= 1) {
-                        const float od = __shfl_xor_sync(0xffffffffu, bd, off);
-                        const int orr = __shfl_xor_sync(0xffffffffu, br, off);
-                        if (orr != 0x7fffffff && (br == 0x7fffffff || od > bd || (od == bd && orr < br))) {
-                            bd = od;
-                            br = orr;
-                        }
-                    }
-                    if (lane == 0) flags[2] = br;
-                }
-                csync();
-                res_target = flags[2];
-                merge_slot = res_target;
-                const uint32_t wr_u = w_s[res_target];
-                res_w = wr_u + 1u;
-                const float wr = static_cast<float>(wr_u);
-                // Eq. (kvr): incremental mean of key and value
-                for (int k = tid; k < D; k += NT) {
-                    mk[k] = fmaf(wr, Kr_g[(size_t)res_target * D + k], kc[k]) / (wr + 1.0f);
-                    mv[k] = fmaf(wr, Vr_g[(size_t)res_target * D + k], vc[k]) / (wr + 1.0f);
-                }
-            }
+            mail->victim_slot = victim_slot;
+            mail->victim_pos = victim_pos;
+            mail->evict = evict ? 1 : 0;
+            mail->s_tok = s_tok;
+            mbar_arrive(&post_bar[mb]);
         }
 
         // ---------------- D3: output ----------------
-        float acc[G][EPL];
+        float2 acc2[G][EP2];
 #pragma unroll
         for (int g = 0; g < G; ++g)
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) acc[g][e] = 0.f;
+            for (int e = 0; e < EP2; ++e) acc2[g][e] = make_float2(0.f, 0.f);
         for (int r0 = 0; r0 < n_live; r0 += R) {
             const uint8_t *tile = wait_full(W_V);
             if (!tile) return;
             const int rows = min(R, n_live - r0);
-            for (int base = warp * RPW; base < rows; base += NW * RPW * UB) {
-                uint4 raw[UB];
+            for (int base = warp * RPW; base < rows; base += NW * RPW * UBV) {
+                uint4 raw[UBV];
 #pragma unroll
-                for (int u = 0; u < UB; ++u) {
+                for (int u = 0; u < UBV; ++u) {
                     const int row = base + u * NW * RPW + sub;
                     raw[u] = row < rows
                                  ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
                                  : make_uint4(0, 0, 0, 0);
                 }
 #pragma unroll
-                for (int u = 0; u < UB; ++u) {
+                for (int u = 0; u < UBV; ++u) {
                     const int row = base + u * NW * RPW + sub;
                     float f[EPL];
                     E::widen(raw[u], f);
+                    float pv[G];
+                    if (row < rows) {
+                        load_group<G>(probs + (r0 + row) * G, pv);
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < G; ++g) pv[g] = 0.f;
+                    }
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
-                        const float pj = row < rows ? probs[g * LS + r0 + row] : 0.f;
+                        const float2 pp = make_float2(pv[g], pv[g]);
 #pragma unroll
-                        for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(pj, f[e], acc[g][e]);
+                        for (int e = 0; e < EP2; ++e)
+                            acc2[g][e] = __ffma2_rn(pp, make_float2(f[2 * e], f[2 * e + 1]), acc2[g][e]);
                     }
                 }
             }
@@ -611,13 +837,14 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
                 const int row = base + sub32;
                 if (row < rows) {
                     const float4 vr = *reinterpret_cast<const float4 *>(tile + row * ROWB32 + l32 * 16);
+                    float pv[G];
+                    load_group<G>(probs + (n_live + r0 + row) * G, pv);
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
-                        const float pj = probs[g * LS + n_live + r0 + row];
-                        acc32[g][0] = fmaf(pj, vr.x, acc32[g][0]);
-                        acc32[g][1] = fmaf(pj, vr.y, acc32[g][1]);
-                        acc32[g][2] = fmaf(pj, vr.z, acc32[g][2]);
-                        acc32[g][3] = fmaf(pj, vr.w, acc32[g][3]);
+                        acc32[g][0] = fmaf(pv[g], vr.x, acc32[g][0]);
+                        acc32[g][1] = fmaf(pv[g], vr.y, acc32[g][1]);
+                        acc32[g][2] = fmaf(pv[g], vr.z, acc32[g][2]);
+                        acc32[g][3] = fmaf(pv[g], vr.w, acc32[g][3]);
                     }
                 }
             }
@@ -628,7 +855,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
         for (int g = 0; g < G; ++g) {
 #pragma unroll
             for (int e = 0; e < EPL; ++e) {
-                float v = acc[g][e];
+                float v = (e & 1) ? acc2[g][e / 2].y : acc2[g][e / 2].x;
 #pragma unroll
                 for (int off = LPR; off < 32; off <<= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
                 if (sub == 0) opart[(warp * G + g) * D + l * EPL + e] = v;
@@ -649,6 +876,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
             }
         }
         csync();
+        if (tid == 0) mbar_arrive(&vdone_bar[mb]);  // the unit's rows may be overwritten now
         {
             const T *vn = reinterpret_cast<const T *>(vn_raw);
             T *out = static_cast<T *>(p.out) + (size_t)ul * G * D;
@@ -656,45 +884,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
                 const int g = k / D, dim = k % D;
                 float sum = 0.f;
                 for (int wv = 0; wv < NW; ++wv) sum += opart[(wv * G + g) * D + dim];
-                sum = fmaf(probs[g * LS + n_ent - 1], E::to_float(vn[dim]), sum);
+                sum = fmaf(probs[(n_ent - 1) * G + g], E::to_float(vn[dim]), sum);
                 out[k] = E::from_float(sum * inv[g]);
             }
-        }
-
-        // ---------------- D6 + D7: write-back (every read of this unit is done) ----------------
-        const bool insert = evict ? (have_victim && victim_slot >= 0) : true;
-        const int ins_slot = evict ? victim_slot : n_live;
-        if (insert) {
-            if (tid < ROWB / 16) {
-                reinterpret_cast<uint4 *>(p.base + d.k_off + (size_t)ins_slot * ROWB)[tid] = kn_raw[tid];
-            } else if (tid < 2 * (ROWB / 16)) {
-                const int k = tid - ROWB / 16;
-                reinterpret_cast<uint4 *>(p.base + d.v_off + (size_t)ins_slot * ROWB)[k] = vn_raw[k];
-            }
-        }
-        if (res_target >= 0) {
-            float *Kr_g = reinterpret_cast<float *>(p.base + d.kr_off);
-            float *Vr_g = reinterpret_cast<float *>(p.base + d.vr_off);
-            for (int k = tid; k < D; k += NT) {
-                Kr_g[(size_t)res_target * D + k] = mk[k];
-                Vr_g[(size_t)res_target * D + k] = mv[k];
-            }
-        }
-        if (tid == 0) {
-            if (insert) {
-                score_g[ins_slot] = s_tok;
-                pos_g[ins_slot] = Tpos;
-            }
-            if (res_target >= 0)
-                reinterpret_cast<uint32_t *>(p.base + d.w_off)[res_target] = res_w;
-            UnitCounters c;
-            c.n_live = n_live + ((!evict) ? 1 : 0);
-            c.n_res = n_res + ((merge_slot == -2) ? 1 : 0);
-            c.T = Tpos + 1;
-            c.pad = 0;
-            *reinterpret_cast<int4 *>(p.counters + d.unit) = *reinterpret_cast<int4 *>(&c);
-            if (p.victim_pos) p.victim_pos[ul] = victim_pos;
-            if (p.merge_slot) p.merge_slot[ul] = merge_slot;
         }
         csync();  // shared scratch is free for the next unit
     }
@@ -702,7 +894,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_fused_kernel(const Deco
 
 template <typename T, int D, int G>
 int launch_one(const DecodeParams &p, int grid, int consumer_warps, cudaStream_t stream) {
-    const int threads = (consumer_warps + 1) * 32;
+    const int threads = (consumer_warps + kExtraWarps) * 32;
     const DecodeSmem L = decode_smem_layout(p.stages, G, D, D * (int)sizeof(T), p.l_stride,
                                             p.br_max_pad, consumer_warps);
     decode_fused_kernel<T, D, G><<<grid, threads, L.total, stream>>>(p);

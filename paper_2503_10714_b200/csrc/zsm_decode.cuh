@@ -5,8 +5,10 @@
 
 namespace zsm {
 
-constexpr int kTileBytes = 16384;      // one ring stage
-constexpr int kMaxConsumerWarps = 16;  // + 1 producer warp
+constexpr int kTileBytes = 16384;     // one ring stage
+constexpr int kMaxConsumerWarps = 8;  // + 1 producer warp + 1 tail warp
+constexpr int kExtraWarps = 2;
+constexpr int kMailFixed = 128;       // bytes of a mailbox before its key, value and count arrays
 
 struct DecodeParams {
     uint8_t *base;               // cache buffer
@@ -29,8 +31,16 @@ struct DecodeParams {
 
 // Shared-memory map of one CTA (byte offsets), computed the same way on host and device.
 struct DecodeSmem {
-    uint32_t ring, bars, flags, probs, qf, kn, vn, w, opart, redf, red64, dots, rows, total;
+    uint32_t ring, bars, flags, probs, qf, mail, opart, redf, red64, total;
+    uint32_t mail_stride;
 };
+
+// A mailbox hands one unit's cache update (residual fill/merge, insertion, counters) from the
+// consumer warps to the tail warp; two of them, used alternately.
+__host__ __device__ inline uint32_t decode_mail_bytes(int row_bytes, int br_max_pad) {
+    const uint32_t b = kMailFixed + 2u * row_bytes + static_cast<uint32_t>(br_max_pad > 0 ? br_max_pad : 4) * 4u;
+    return (b + 127u) & ~127u;
+}
 
 __host__ __device__ inline DecodeSmem decode_smem_layout(int stages, int G, int D, int row_bytes,
                                                          int l_stride, int br_max_pad,
@@ -43,18 +53,15 @@ __host__ __device__ inline DecodeSmem decode_smem_layout(int stages, int G, int 
         return at;
     };
     L.ring = take(static_cast<uint32_t>(stages) * kTileBytes);
-    L.bars = take(static_cast<uint32_t>(stages) * 16u);
+    L.bars = take((2u * static_cast<uint32_t>(stages) + 6u) * 8u);
     L.flags = take(64u);
     L.probs = take(static_cast<uint32_t>(G) * l_stride * 4u);
     L.qf = take(static_cast<uint32_t>(G) * D * 4u);
-    L.kn = take(static_cast<uint32_t>(row_bytes));
-    L.vn = take(static_cast<uint32_t>(row_bytes));
-    L.w = take(static_cast<uint32_t>(br_max_pad > 0 ? br_max_pad : 4) * 4u);
+    L.mail_stride = decode_mail_bytes(row_bytes, br_max_pad);
+    L.mail = take(2u * L.mail_stride);
     L.opart = take(static_cast<uint32_t>(consumer_warps) * G * D * 4u);
     L.redf = take(2u * kMaxConsumerWarps * 8u * 4u);
     L.red64 = take(kMaxConsumerWarps * 16u);
-    L.dots = take(static_cast<uint32_t>(br_max_pad > 0 ? br_max_pad : 4) * 4u);
-    L.rows = take(4u * D * 4u);
     L.total = o;
     return L;
 }
