@@ -68,6 +68,7 @@ struct Elem;
 template <>
 struct Elem<float> {
     static constexpr int EPL = 4;
+    static constexpr bool kIsBf16 = false;
     __device__ static __forceinline__ void widen(const uint4 &raw, float (&f)[4]) {
         f[0] = __uint_as_float(raw.x);
         f[1] = __uint_as_float(raw.y);
@@ -81,6 +82,7 @@ struct Elem<float> {
 template <>
 struct Elem<__half> {
     static constexpr int EPL = 8;
+    static constexpr bool kIsBf16 = false;
     __device__ static __forceinline__ void widen(const uint4 &raw, float (&f)[8]) {
         const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
 #pragma unroll
@@ -97,6 +99,7 @@ struct Elem<__half> {
 template <>
 struct Elem<__nv_bfloat16> {
     static constexpr int EPL = 8;
+    static constexpr bool kIsBf16 = true;
     __device__ static __forceinline__ void widen(const uint4 &raw, float (&f)[8]) {
         const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -149,6 +152,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
+// The same test, but the thread may stay suspended for up to `hint_ns` (a hint; the hardware
+// caps it) or until the phase completes, instead of returning at once: a waiting warp then
+// issues a poll now and then rather than spinning.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t *bar, uint32_t parity,
+                                                      uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -161,6 +182,7 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // whose phase has completed always returns true, whatever the abort flag says,
 // so every thread of a CTA stops at the same point of the tile sequence.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr uint32_t kSuspendHintNs = 20000u;        // per poll
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity,
                                                   volatile int32_t *abort_flag, int32_t *status,
@@ -169,9 +191,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
     const uint64_t t0 = global_timer_ns();
     uint32_t polls = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_suspend(bar, parity, kSuspendHintNs)) return true;
         ++polls;
-        if ((polls & 63u) == 0u) {
+        if ((polls & 7u) == 0u) {
             if (*abort_flag) return false;
             if (global_timer_ns() - t0 > kWaitLimitNs) {
                 dev_set_status(status, DEV_ERR_TIMEOUT, where, static_cast<int32_t>(blockIdx.x));

@@ -56,6 +56,11 @@ __device__ __forceinline__ float group_sum(float v) {
     return v;
 }
 
+template <bool B>
+struct BoolC {
+    static constexpr bool value = B;
+};
+
 __host__ __device__ constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
 
 // Sums each of the N values over the LG lanes of a group with a transposing butterfly: while
@@ -148,6 +153,26 @@ __device__ __forceinline__ void load4(const T *p, float (&f)[4]) {
     }
 }
 
+// One m16n8k16 tensor-core step with fp32 accumulation: c += A(16 x 16, row-major) * B(16 x 8).
+// a0..a3 and b0, b1 are packed pairs of 16-bit elements in the instruction's fragment order.
+template <typename T>
+__device__ __forceinline__ void mma_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                            uint32_t a3, uint32_t b0, uint32_t b1) {
+    if constexpr (sizeof(T) == 2 && Elem<T>::kIsBf16) {
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+            "{%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    } else {
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+            "{%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+}
+
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const DecodeParams p) {
     using E = Elem<T>;
@@ -171,6 +196,10 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
     constexpr int UBV = G <= 4 ? 4 : 2;       // same, output pass
     constexpr int NV = G * UBK;               // partial dot products a lane carries
     constexpr int NF = NV > LPR ? NV / LPR : 1;
+    // 16-bit storage: the logits pass runs on the tensor cores, 16 slots x 8 query heads per step
+    constexpr bool kMma = sizeof(T) == 2;
+    constexpr int SEG = ROWB / 64;            // 64-byte column segments of a token row
+    constexpr int RB = R / 16;                // 16-row blocks per tile
 
     extern __shared__ __align__(128) uint8_t smem[];
     const int NW = (blockDim.x >> 5) - kExtraWarps;  // consumer warps
@@ -496,6 +525,10 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
     };
     auto csync = [&]() { named_bar_sync(1, NT); };
 
+    // a full tile needs no row checks when the warps' row groups tile it exactly
+    const bool full_k = (R % (NW * RPW * UBK)) == 0;
+    const bool full_v = (R % (NW * RPW * UBV)) == 0;
+    const int rb_step = RB % NW;  // how far a tile's 16-row blocks advance the round-robin
     // where this lane's sums land after the transposing reduction of the logits pass
     const int tr_idx = treduce_index<NV, LPR>(l);
     const bool tr_writer = (NV >= LPR) || ((l & (LPR / (NV < LPR ? NV : LPR) - 1)) == 0);
@@ -527,14 +560,30 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
         const int Tpos = cnt.z;
         const int n_ent = n_live + n_res + 1;
 
-        float2 q2[G][EP2];
+        // query operands of the logits pass: packed fp32 pairs for the FMA form, or the B
+        // fragments (head n = lane / 4; heads >= G are zero) for the tensor-core form
+        float2 q2[kMma ? 1 : G][kMma ? 1 : EP2];
+        uint32_t qb[kMma ? SEG : 1][4];
+        if constexpr (kMma) {
+            const int gq = lane >> 2, tig = lane & 3;
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const uint4 raw = *reinterpret_cast<const uint4 *>(h + HDR_Q + g * ROWB + l * 16);
-            float f[EPL];
-            E::widen(raw, f);
+            for (int j = 0; j < SEG; ++j) {
+                uint4 t = make_uint4(0, 0, 0, 0);
+                if (gq < G) t = *reinterpret_cast<const uint4 *>(h + HDR_Q + gq * ROWB + j * 64 + tig * 16);
+                qb[j][0] = t.x;
+                qb[j][1] = t.y;
+                qb[j][2] = t.z;
+                qb[j][3] = t.w;
+            }
+        } else {
 #pragma unroll
-            for (int e = 0; e < EP2; ++e) q2[g][e] = make_float2(f[2 * e], f[2 * e + 1]);
+            for (int g = 0; g < G; ++g) {
+                const uint4 raw = *reinterpret_cast<const uint4 *>(h + HDR_Q + g * ROWB + l * 16);
+                float f[EPL];
+                E::widen(raw, f);
+#pragma unroll
+                for (int e = 0; e < EP2; ++e) q2[g][e] = make_float2(f[2 * e], f[2 * e + 1]);
+            }
         }
         {
             const T *qs = reinterpret_cast<const T *>(h + HDR_Q);
@@ -555,43 +604,83 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
         release();
 
         // ---------------- D1: logits of the token slots ----------------
+        int kturn = 0;
         for (int r0 = 0; r0 < n_live; r0 += R) {
             const uint8_t *tile = wait_full(W_K);
             if (!tile) return;
             const int rows = min(R, n_live - r0);
-            for (int base = warp * RPW; base < rows; base += NW * RPW * UBK) {
-                uint4 raw[UBK];
+            if constexpr (kMma) {
+                // Blocks of 16 rows go round the warps.  A thread reads 16 bytes of rows
+                // gq and gq + 8 per 64-byte segment; the contraction index is permuted the
+                // same way on both operands, so each 16-byte read feeds two steps.
+                const int gq = lane >> 2, tig = lane & 3;
+                int rb_first = warp - kturn;  // kturn: this tile's first block, modulo NW
+                if (rb_first < 0) rb_first += NW;
+                for (int rb = rb_first; rb < RB && rb * 16 < rows; rb += NW) {
+                    const uint8_t *pa = tile + (rb * 16 + gq) * ROWB + tig * 16;
+                    float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int u = 0; u < UBK; ++u) {
-                    const int row = base + u * NW * RPW + sub;
-                    raw[u] = row < rows
-                                 ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
-                                 : make_uint4(0, 0, 0, 0);
-                }
-                float v[NV];
-#pragma unroll
-                for (int u = 0; u < UBK; ++u) {
-                    float f[EPL];
-                    E::widen(raw[u], f);
-#pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        float2 a = make_float2(0.f, 0.f);
-#pragma unroll
-                        for (int e = 0; e < EP2; ++e)
-                            a = __ffma2_rn(q2[g][e], make_float2(f[2 * e], f[2 * e + 1]), a);
-                        v[u * G + g] = a.x + a.y;
+                    for (int j = 0; j < SEG; ++j) {
+                        const uint4 ra = *reinterpret_cast<const uint4 *>(pa + j * 64);
+                        const uint4 rc = *reinterpret_cast<const uint4 *>(pa + 8 * ROWB + j * 64);
+                        mma_16x8x16<T>(c0, ra.x, rc.x, ra.y, rc.y, qb[j][0], qb[j][1]);
+                        mma_16x8x16<T>(c1, ra.z, rc.z, ra.w, rc.w, qb[j][2], qb[j][3]);
+                    }
+                    const int n0 = tig * 2;  // query heads n0, n0 + 1 of rows gq and gq + 8
+                    if (n0 < G) {
+                        const int ra_ = rb * 16 + gq, rc_ = ra_ + 8;
+                        float *pr = probs + (r0 + ra_) * G + n0;
+                        if (ra_ < rows) {
+                            pr[0] = (c0[0] + c1[0]) * p.scale;
+                            if (G > 1) pr[1] = (c0[1] + c1[1]) * p.scale;
+                        }
+                        if (rc_ < rows) {
+                            pr[8 * G] = (c0[2] + c1[2]) * p.scale;
+                            if (G > 1) pr[8 * G + 1] = (c0[3] + c1[3]) * p.scale;
+                        }
                     }
                 }
-                treduce<NV, LPR>(v, l);
-                if (tr_writer) {
-#pragma unroll
-                    for (int k = 0; k < NF; ++k) {
-                        const int id = tr_idx + k;
-                        const int u = id / G, g = id % G;
-                        const int row = base + u * NW * RPW + sub;
-                        if (row < rows) probs[(r0 + row) * G + g] = v[k] * p.scale;
+                kturn += rb_step;
+                if (kturn >= NW) kturn -= NW;
+            } else {
+                auto k_rows = [&](auto full) {
+                    constexpr bool FULL = decltype(full)::value;  // every row of the pass exists
+                    for (int base = warp * RPW; base < rows; base += NW * RPW * UBK) {
+                        uint4 raw[UBK];
+    #pragma unroll
+                        for (int u = 0; u < UBK; ++u) {
+                            const int row = base + u * NW * RPW + sub;
+                            raw[u] = (FULL || row < rows)
+                                         ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
+                                         : make_uint4(0, 0, 0, 0);
+                        }
+                        float v[NV];
+    #pragma unroll
+                        for (int u = 0; u < UBK; ++u) {
+                            float f[EPL];
+                            E::widen(raw[u], f);
+    #pragma unroll
+                            for (int g = 0; g < G; ++g) {
+                                float2 a = make_float2(0.f, 0.f);
+    #pragma unroll
+                                for (int e = 0; e < EP2; ++e)
+                                    a = __ffma2_rn(q2[g][e], make_float2(f[2 * e], f[2 * e + 1]), a);
+                                v[u * G + g] = a.x + a.y;
+                            }
+                        }
+                        treduce<NV, LPR>(v, l);
+                        if (tr_writer) {
+    #pragma unroll
+                            for (int k = 0; k < NF; ++k) {
+                                const int id = tr_idx + k;
+                                const int u = id / G, g = id % G;
+                                const int row = base + u * NW * RPW + sub;
+                                if (FULL || row < rows) probs[(r0 + row) * G + g] = v[k] * p.scale;
+                            }
+                        }
                     }
-                }
+                };
+                if (rows == R && full_k) k_rows(BoolC<true>{}); else k_rows(BoolC<false>{});
             }
             release();
         }
@@ -792,36 +881,40 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
             const uint8_t *tile = wait_full(W_V);
             if (!tile) return;
             const int rows = min(R, n_live - r0);
-            for (int base = warp * RPW; base < rows; base += NW * RPW * UBV) {
-                uint4 raw[UBV];
+            auto v_rows = [&](auto full) {
+                constexpr bool FULL = decltype(full)::value;
+                for (int base = warp * RPW; base < rows; base += NW * RPW * UBV) {
+                    uint4 raw[UBV];
 #pragma unroll
-                for (int u = 0; u < UBV; ++u) {
-                    const int row = base + u * NW * RPW + sub;
-                    raw[u] = row < rows
-                                 ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
-                                 : make_uint4(0, 0, 0, 0);
-                }
-#pragma unroll
-                for (int u = 0; u < UBV; ++u) {
-                    const int row = base + u * NW * RPW + sub;
-                    float f[EPL];
-                    E::widen(raw[u], f);
-                    float pv[G];
-                    if (row < rows) {
-                        load_group<G>(probs + (r0 + row) * G, pv);
-                    } else {
-#pragma unroll
-                        for (int g = 0; g < G; ++g) pv[g] = 0.f;
+                    for (int u = 0; u < UBV; ++u) {
+                        const int row = base + u * NW * RPW + sub;
+                        raw[u] = (FULL || row < rows)
+                                     ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
+                                     : make_uint4(0, 0, 0, 0);
                     }
 #pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        const float2 pp = make_float2(pv[g], pv[g]);
+                    for (int u = 0; u < UBV; ++u) {
+                        const int row = base + u * NW * RPW + sub;
+                        float f[EPL];
+                        E::widen(raw[u], f);
+                        float pv[G];
+                        if (FULL || row < rows) {
+                            load_group<G>(probs + (r0 + row) * G, pv);
+                        } else {
 #pragma unroll
-                        for (int e = 0; e < EP2; ++e)
-                            acc2[g][e] = __ffma2_rn(pp, make_float2(f[2 * e], f[2 * e + 1]), acc2[g][e]);
+                            for (int g = 0; g < G; ++g) pv[g] = 0.f;
+                        }
+#pragma unroll
+                        for (int g = 0; g < G; ++g) {
+                            const float2 pp = make_float2(pv[g], pv[g]);
+#pragma unroll
+                            for (int e = 0; e < EP2; ++e)
+                                acc2[g][e] = __ffma2_rn(pp, make_float2(f[2 * e], f[2 * e + 1]), acc2[g][e]);
+                        }
                     }
                 }
-            }
+            };
+            if (rows == R && full_v) v_rows(BoolC<true>{}); else v_rows(BoolC<false>{});
             release();
         }
         float acc32[G][4];
