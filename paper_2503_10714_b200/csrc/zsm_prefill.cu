@@ -8,8 +8,9 @@
 //   P2  the latest B_p positions are kept as they are (Sec. 3.2)
 //   P3  prefill_select     of the rest, the B_c highest (score, position) stay: radix
 //                          select of the eviction threshold, then ordered compaction
-//   P4  prefill_merge      evicted tokens, ascending position, fill-or-merge into the
-//                          residual slots (Alg. 1 l.12-16, Eq. (hatr), (kvr))
+//   P4  prefill_merge[_reg] evicted tokens, ascending position, fill-or-merge into the
+//                          residual slots (Alg. 1 fill/merge branch, Eq. (hatr), (kvr));
+//                          the register form holds the merged keys in registers (B_r <= 128)
 //   P5  prefill_gather     survivors' rows, scores and positions into the unit's slots
 #include "zsm_prefill.cuh"
 
@@ -439,6 +440,216 @@ __global__ void __launch_bounds__(kMergeWarps * 32) prefill_merge_kernel(const P
 }
 
 // ---------------------------------------------------------------------------
+// P4, register form (B_r <= 32 * RT): one CTA of 256 threads per unit.  Thread (row, seg)
+// keeps D/8 consecutive floats of RT merged keys in registers (rows tid/8 + 32*j, segment
+// tid%8); merged values, which only the chosen row's threads touch, stay in shared memory.
+// Per evicted token: every thread dots its key segments with the token's, three shuffles
+// finish the dot products, a shuffle/shared-memory argmax picks the slot, the slot's eight
+// threads apply Eq. (kvr).  One barrier per token; evicted rows arrive through a cp.async
+// ring several tokens ahead.
+// ---------------------------------------------------------------------------
+constexpr int kRegMergeThreads = 256;
+constexpr int kRegMergePF = 10;  // ring slots; a slot is refilled two tokens after its use
+constexpr int kRegMergeIdx = (kMergeIB + kRegMergePF + 3) & ~3;  // staged positions, padded so
+                                                                 // the ring after them stays
+                                                                 // 16-byte aligned for cp.async
+
+template <typename T, int D, int RT>
+__global__ void __launch_bounds__(kRegMergeThreads) prefill_merge_reg_kernel(const PrefillParams p) {
+    using E = Elem<T>;
+    constexpr int ROWB = D * (int)sizeof(T);
+    constexpr int CPR = ROWB / 16;   // 16-byte chunks per row
+    constexpr int SEG = D / 8;       // floats per thread and row
+    constexpr int PF = kRegMergePF;
+    static_assert(2 * CPR <= kRegMergeThreads, "one cp.async per thread covers a K and a V row");
+    static_assert((32 * 4 + kRegMergeIdx * 4) % 16 == 0 && (D * 4) % 16 == 0,
+                  "the ring of 16-byte copies starts on a 16-byte boundary");
+    extern __shared__ __align__(16) uint8_t smraw[];
+
+    const int ul = blockIdx.x;
+    const UnitDesc d = p.desc[ul];
+    const int Br = d.Br;
+    const int T_len = p.T;
+    const int n_ev = reinterpret_cast<const int32_t *>(p.ws + p.wl.counts)[ul * 4];
+    const int32_t *evl = reinterpret_cast<const int32_t *>(p.ws + p.wl.evict_list) + (size_t)ul * T_len;
+    int32_t *targets = p.dbg_targets ? p.dbg_targets + (size_t)ul * T_len : nullptr;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int seg = tid & 7, row0 = tid >> 3;
+
+    if (Br == 0) {
+        if (targets)
+            for (int i = tid; i < n_ev; i += blockDim.x) targets[i] = -1;  // dropped (Sec. 3.2)
+        return;
+    }
+    float *Vr_s = reinterpret_cast<float *>(smraw);                       // [Br][D]
+    float *best_v = Vr_s + (size_t)Br * D;                                // [2][8] per-warp maxima
+    int32_t *best_r = reinterpret_cast<int32_t *>(best_v + 16);           // [2][8]
+    int32_t *idx_s = best_r + 16;                                         // [kRegMergeIdx]
+    uint8_t *ring = reinterpret_cast<uint8_t *>(idx_s + kRegMergeIdx);    // [PF][2][ROWB]
+
+    const uint8_t *Kg = static_cast<const uint8_t *>(p.K) + (size_t)ul * T_len * ROWB;
+    const uint8_t *Vg = static_cast<const uint8_t *>(p.V) + (size_t)ul * T_len * ROWB;
+
+    float kr[RT][SEG];  // this thread's segments of the merged keys
+    float wr[RT];       // their fusion counts (kept by all eight threads of a row)
+#pragma unroll
+    for (int j = 0; j < RT; ++j) {
+        wr[j] = 0.f;
+#pragma unroll
+        for (int e = 0; e < SEG; ++e) kr[j][e] = 0.f;
+    }
+
+    int i0 = 0;  // idx_s[j] = evl[i0 + j]
+    auto stage_indices = [&](int start) {
+        for (int j = tid; j < kRegMergeIdx; j += blockDim.x)
+            idx_s[j] = (start + j < n_ev) ? evl[start + j] : 0;
+    };
+    auto issue = [&](int i) {  // fetch evicted token i's rows into ring slot i % PF
+        if (i < n_ev && tid < 2 * CPR) {
+            const int which = tid / CPR, c = tid % CPR;
+            const int t = idx_s[i - i0];
+            const uint8_t *src = (which ? Vg : Kg) + (size_t)t * ROWB + c * 16;
+            cp_async16(ring + ((size_t)(i % PF) * 2 + which) * ROWB + c * 16, src);
+        }
+        cp_async_commit();
+    };
+    auto load_seg = [&](const uint8_t *rowp, float (&f)[SEG]) {  // 16-byte loads, widened
+        const uint4 *src = reinterpret_cast<const uint4 *>(rowp + seg * SEG * sizeof(T));
+#pragma unroll
+        for (int c = 0; c < SEG / E::EPL; ++c) {
+            float t[E::EPL];
+            E::widen(src[c], t);
+#pragma unroll
+            for (int e = 0; e < E::EPL; ++e) f[c * E::EPL + e] = t[e];
+        }
+    };
+
+    stage_indices(0);
+    __syncthreads();
+    for (int i = 0; i < PF - 2; ++i) issue(i);  // tokens 0 .. PF-3 in flight
+    cp_async_wait<PF - 3>();                    // token 0 has landed
+    __syncthreads();
+
+    for (int i = 0; i < n_ev; ++i) {
+        // ring slot of token i-2 is free (its last readers passed the barrier of token i-1)
+        issue(i + PF - 2);
+        const uint8_t *kc_row = ring + ((size_t)(i % PF) * 2 + 0) * ROWB;
+        const uint8_t *vc_row = ring + ((size_t)(i % PF) * 2 + 1) * ROWB;
+        float kc[SEG];
+        load_seg(kc_row, kc);
+        int target;
+        if (i < Br) {
+            target = i;  // Alg. 1: a free residual slot takes the token as it is
+        } else {
+            // Eq. (hatr): raw dot products, ties to the lowest slot
+            float bv = -INFINITY;
+            int br = 0x7fffffff;
+#pragma unroll
+            for (int j = 0; j < RT; ++j) {
+                float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                for (int e = 0; e < SEG; e += 2) {
+                    a0 = fmaf(kr[j][e], kc[e], a0);
+                    a1 = fmaf(kr[j][e + 1], kc[e + 1], a1);
+                }
+                float dot = a0 + a1;
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                const int r = row0 + 32 * j;
+                if (r < Br && (br == 0x7fffffff || dot > bv)) {
+                    bv = dot;
+                    br = r;
+                }
+            }
+#pragma unroll
+            for (int off = 8; off <= 16; off <<= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                const int orr = __shfl_xor_sync(0xffffffffu, br, off);
+                if (orr != 0x7fffffff && (br == 0x7fffffff || ov > bv || (ov == bv && orr < br))) {
+                    bv = ov;
+                    br = orr;
+                }
+            }
+            if (lane == 0) {
+                best_v[(i & 1) * 8 + warp] = bv;
+                best_r[(i & 1) * 8 + warp] = br;
+            }
+            target = -1;
+        }
+        // token i+1 must have landed before the barrier that publishes it
+        cp_async_wait<PF - 3>();
+        __syncthreads();
+        if (target < 0) {
+            float bv = best_v[(i & 1) * 8];
+            int br = best_r[(i & 1) * 8];
+#pragma unroll
+            for (int wv = 1; wv < 8; ++wv) {
+                const float ov = best_v[(i & 1) * 8 + wv];
+                const int orr = best_r[(i & 1) * 8 + wv];
+                if (orr != 0x7fffffff && (br == 0x7fffffff || ov > bv || (ov == bv && orr < br))) {
+                    bv = ov;
+                    br = orr;
+                }
+            }
+            target = br;
+        }
+        // Eq. (kvr) on the chosen row, by its eight threads
+#pragma unroll
+        for (int j = 0; j < RT; ++j) {
+            if (row0 + 32 * j == target) {
+                const float w = wr[j];
+                const float dn = w + 1.0f;
+                // one correctly rounded reciprocal instead of 2*SEG divisions on the chain's
+                // critical path (the divisions alone were two thirds of a merge's time)
+                const float rdn = __frcp_rn(dn);
+                float vc[SEG];
+                load_seg(vc_row, vc);
+                float *vr = Vr_s + (size_t)target * D + seg * SEG;
+#pragma unroll
+                for (int e = 0; e < SEG; ++e) {
+                    kr[j][e] = (w == 0.f) ? kc[e] : fmaf(w, kr[j][e], kc[e]) * rdn;
+                    vr[e] = (w == 0.f) ? vc[e] : fmaf(w, vr[e], vc[e]) * rdn;
+                }
+                wr[j] = dn;
+                if (seg == 0 && targets) targets[i] = (i < Br) ? -2 : target;
+            }
+        }
+        if (i + 1 - i0 == kMergeIB && i + 1 < n_ev) {
+            // next block of positions; tokens up to i + PF - 2 were issued from the old block,
+            // whose tail (PF extra entries) covers them
+            __syncthreads();
+            i0 = i + 1;
+            stage_indices(i0);
+            __syncthreads();
+        }
+    }
+    cp_async_wait<0>();
+
+    const int n_res = min(Br, n_ev);
+    float *Kr_g = reinterpret_cast<float *>(p.base + d.kr_off);
+    float *Vr_g = reinterpret_cast<float *>(p.base + d.vr_off);
+    uint32_t *w_g = reinterpret_cast<uint32_t *>(p.base + d.w_off);
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < RT; ++j) {
+        const int r = row0 + 32 * j;
+        if (r < n_res) {
+#pragma unroll
+            for (int e = 0; e < SEG; ++e) Kr_g[(size_t)r * D + seg * SEG + e] = kr[j][e];
+            if (seg == 0) w_g[r] = static_cast<uint32_t>(wr[j]);
+        }
+    }
+    for (int k = tid; k < n_res * D; k += blockDim.x) Vr_g[k] = Vr_s[k];
+}
+
+template <typename T, int D>
+size_t merge_reg_smem_bytes(int Br) {
+    return (size_t)Br * D * 4 + 32 * 4 + (size_t)kRegMergeIdx * 4 +
+           (size_t)kRegMergePF * 2 * D * sizeof(T);
+}
+
+// ---------------------------------------------------------------------------
 // P5: survivors into the unit's slots, ascending position; one warp per row.
 // ---------------------------------------------------------------------------
 template <typename T, int D>
@@ -498,8 +709,16 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
         scores = reinterpret_cast<const float *>(p.ws + p.wl.scores);
     }
     prefill_select_kernel<<<p.units, 1024, 0, stream>>>(p, scores);
-    prefill_merge_kernel<T, D><<<p.units, kMergeWarps * 32,
-                                 merge_smem_bytes<D>(max_br, D * (int)sizeof(T)), stream>>>(p);
+    // the residual chain: merged keys in registers when the layer's largest B_r allows it
+    if (max_br <= 32)
+        prefill_merge_reg_kernel<T, D, 1><<<p.units, kRegMergeThreads, merge_reg_smem_bytes<T, D>(max_br), stream>>>(p);
+    else if (max_br <= 64)
+        prefill_merge_reg_kernel<T, D, 2><<<p.units, kRegMergeThreads, merge_reg_smem_bytes<T, D>(max_br), stream>>>(p);
+    else if (max_br <= 128)
+        prefill_merge_reg_kernel<T, D, 4><<<p.units, kRegMergeThreads, merge_reg_smem_bytes<T, D>(max_br), stream>>>(p);
+    else
+        prefill_merge_kernel<T, D><<<p.units, kMergeWarps * 32,
+                                     merge_smem_bytes<D>(max_br, D * (int)sizeof(T)), stream>>>(p);
     // the largest unit bounds the gather grid; rows past a unit's survivors return at once
     const int max_rows = p.max_cap < p.T ? p.max_cap : p.T;
     prefill_gather_kernel<T, D><<<dim3((max_rows + 7) / 8, p.units), 256, 0, stream>>>(p, scores);
@@ -515,6 +734,15 @@ int prepare_all() {
     e = cudaFuncSetAttribute(prefill_merge_kernel<T, D>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)merge_smem_bytes<D>(prefill_max_residual(D), D * (int)sizeof(T)));
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = cudaFuncSetAttribute(prefill_merge_reg_kernel<T, D, 1>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_reg_smem_bytes<T, D>(32));
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = cudaFuncSetAttribute(prefill_merge_reg_kernel<T, D, 2>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_reg_smem_bytes<T, D>(64));
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = cudaFuncSetAttribute(prefill_merge_reg_kernel<T, D, 4>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_reg_smem_bytes<T, D>(128));
     return static_cast<int>(e);
 }
 

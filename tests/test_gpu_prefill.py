@@ -80,6 +80,21 @@ def test_prompt_pass_degenerate_budgets(zb, oracle, budgets):
         cache.close()
 
 
+@pytest.mark.parametrize("br", [3, 33, 100, 150])
+def test_residual_pool_sizes(zb, oracle, br):
+    """Residual pools on both sides of the sizes at which the merge kernel changes form: merged
+    keys in registers with one, two or four rows per thread (B_r <= 32, 64, 128), in shared
+    memory beyond that."""
+    w = wl.Workload("pool", 1, 1, 2, 2, 128, "f16", 1500, 0, 16, None, 25)
+    cache = GpuCache(zb, w, [[40, 64]], [[60, 90]], [[br, max(1, br // 2)]])
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats)
+        assert cache.status() == 0 and stats.merges > 2000
+    finally:
+        cache.close()
+
+
 def test_supplied_scores_with_exact_ties(zb, oracle):
     """Scores given by the caller, drawn from four values only: the selection is decided by
     the position rule almost everywhere and must match the oracle bit for bit (no near tie
