@@ -30,6 +30,7 @@ namespace zsm {
 namespace {
 
 constexpr int kMaxThreads = (kMaxConsumerWarps + kExtraWarps) * 32;
+constexpr int kMaxDynamicSmem = 232448;  // 227 KiB, the opt-in limit per CTA on sm_100
 
 // "where" codes recorded with a timeout
 enum : int32_t {
@@ -996,8 +997,11 @@ int launch_one(const DecodeParams &p, int grid, int consumer_warps, cudaStream_t
 
 template <typename T, int D, int G>
 int prepare_one(int smem_bytes, int threads, int *max_ctas) {
+    // The limit belongs to the kernel, not to a cache: caches of one shape but different budgets
+    // ask for different amounts, so it is raised to the most any of them can ask for.
     cudaError_t e = cudaFuncSetAttribute(decode_fused_kernel<T, D, G>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kMaxDynamicSmem);
     if (e != cudaSuccess) return static_cast<int>(e);
     int n = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_fused_kernel<T, D, G>, threads,

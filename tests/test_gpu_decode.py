@@ -230,3 +230,21 @@ def test_argument_errors_reach_the_caller(zb):
         assert e.value.status == zb.ZSM_ERR_UNSUPPORTED
     finally:
         c.close()
+
+
+def test_caches_of_one_shape_and_different_budgets_coexist(zb):
+    """Two live caches that use the same kernel but need different amounts of shared memory:
+    creating the second must not lower the launch limit the first one needs."""
+    w = wl.Workload("coexist", 1, 1, 2, 2, 128, "f16", 0, 0, 0, None, 18)
+    small = GpuCache(zb, w, np.full((1, 2), 8), np.full((1, 2), 8), np.full((1, 2), 1))
+    big = GpuCache(zb, w, np.full((1, 2), 100), np.full((1, 2), 15000), np.full((1, 2), 4))
+    try:
+        # the large weight array leaves room for fewer ring stages: the cache created last asks
+        # for less shared memory than the one created first
+        assert zb.zsm_decode_launch_info(big.h, -1)[2] < zb.zsm_decode_launch_info(small.h, -1)[2]
+        q, k, v = (t.cuda() for t in wl.decode_inputs(w, 0))
+        for c in (small, big, small, big):
+            c.decode(q, k, v)
+        assert big.status() == 0 and small.status() == 0
+    finally:
+        big.close(), small.close()

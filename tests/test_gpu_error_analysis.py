@@ -1,0 +1,22 @@
+"""The paper's numerical error analysis (Sec. 4.3) on synthetic heavy-hitter data: at 50, 20,
+10 and 5 % cache the attention output with residual merging is closer to full attention than
+with pure eviction.  The paper gives neither data nor protocol, so the ordering is what is
+checked, not its printed values."""
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+def test_merging_beats_eviction_at_every_ratio():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2503_10714_b200 import error_analysis
+    res = error_analysis.run(prompt_len=2048, steps=64)
+    print(res)
+    for ratio, r in res.items():
+        assert 0.0 < r["merge"] < r["evict"], f"ratio {ratio}: merge {r['merge']:.3e} evict {r['evict']:.3e}"
+    # less cache, more error, for both policies
+    ratios = sorted(res, reverse=True)
+    for a, b in zip(ratios, ratios[1:]):
+        assert res[a]["evict"] < res[b]["evict"] and res[a]["merge"] < res[b]["merge"]
