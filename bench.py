@@ -218,6 +218,48 @@ def oracle_sample(w, K, V, Qw, bp, bc, br, steps, layer=0):
     return dt, len(jobs), threads
 
 
+# ----------------------------------------------------------------------------- FullKV leg
+def fullkv_comparator(zb, w, dev, u, stream, budget_bytes=60e9, steps=10):
+    """Decode attention over the UNCOMPRESSED prompt KV of the same workload (what the paper's
+    FullKV baseline does per step, cache path only), timed with CUDA events.  As many layers as
+    fit in `budget_bytes` are held at once; the step time is scaled to the full stack by layers
+    (layers are independent and equal)."""
+    e = 2
+    per_layer = 2 * w.batch * w.n_kv_heads * w.prompt_len * w.head_dim * e
+    n_l = int(max(1, min(w.n_layers, budget_bytes // per_layer)))
+    upl = w.batch * w.n_kv_heads
+    K = torch.empty(n_l * upl, w.prompt_len, w.head_dim, dtype=w.torch_dtype, device=dev)
+    V = torch.empty_like(K)
+    for layer in range(n_l):
+        Kp, Vp, _ = wl.prompt(w, layer, dev, u)
+        K[layer * upl:(layer + 1) * upl] = Kp.reshape(upl, w.prompt_len, w.head_dim)
+        V[layer * upl:(layer + 1) * upl] = Vp.reshape(upl, w.prompt_len, w.head_dim)
+        del Kp, Vp
+    q_all, _, _ = wl.decode_inputs(w, 0, dev, u)
+    q = q_all[:n_l].reshape(n_l * upl, w.group, w.head_dim).contiguous()
+    out = torch.empty_like(q)
+    ws = torch.empty(zb.zsm_fullkv_workspace_bytes(n_l * upl, w.group, w.head_dim, w.prompt_len),
+                     dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        zb.zsm_fullkv_decode(K, V, q, out, ws)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(steps):
+        zb.zsm_fullkv_decode(K, V, q, out, ws)
+    ev1.record(stream)
+    ev1.synchronize()
+    if zb.zsm_fullkv_status(ws) != 0:
+        raise RuntimeError("device status after the uncompressed-cache comparator is not OK")
+    ms_timed = ev0.elapsed_time(ev1) / steps
+    nbytes = n_l * (per_layer + upl * 2 * w.group * w.head_dim * e)
+    ms_full = ms_timed * w.n_layers / n_l
+    return {"what": "decode attention over the uncompressed prompt KV, same kernels' ring and tensor-core logits",
+            "context": w.prompt_len, "layers_timed": n_l, "ms_per_step": ms_full,
+            "tokens_per_s": w.batch / (ms_full * 1e-3), "achieved_gbs": nbytes / (ms_timed * 1e-3) / 1e9,
+            "bytes_per_step_all_layers": int(nbytes * w.n_layers / n_l)}
+
+
 # ----------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -229,6 +271,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--cpu-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fullkv", action="store_true",
+                    help="skip the uncompressed-cache comparator (same box, same shapes)")
     ap.add_argument("--layers", type=int, default=0,
                     help="run a shallower stack than the workload names (profiling captures only; "
                          "the reported config says so)")
@@ -335,6 +379,10 @@ def main():
         zb.zsm_cache_free(cache)
         return
 
+    fullkv = None
+    if world == 1 and not args.no_fullkv and w.dtype != "f32":
+        fullkv = fullkv_comparator(zb, w, dev, u, stream)
+
     # ---- roofline of the dominant (only) kernel of the timed region ----
     n_live = (bp + bc).astype(np.int64)      # every unit is full after a 54k prompt
     n_res = br.astype(np.int64)
@@ -373,6 +421,9 @@ def main():
         "prompt_pass": {"ms_total": prefill_ms, "ms_per_layer": prefill_ms / w.n_layers,
                         "window": w.window},
     }
+    if fullkv is not None:
+        fullkv["compressed_speedup"] = fullkv["ms_per_step"] / ms_per_step
+        line["fullkv"] = fullkv
     if world == 1 and not args.no_cpu_baseline and sample_prompt is not None:
         dt, n_sampled, threads = oracle_sample(w, *sample_prompt, bp, bc, br, args.cpu_steps)
         n_units = w.n_layers * w.batch * w.n_kv_heads

@@ -188,6 +188,26 @@ zsm_status_t zsm_decode_step_host(zsm_cache_t *c, int32_t layer, const void *q_h
                                   void *out_host, void *staging, size_t staging_bytes,
                                   zsm_stream_t stream);
 
+/* Decode attention over an UNCOMPRESSED cache [Eq. (att_score), Sec. 3.1]: what the paper's
+ * FullKV baseline computes per step, for the cache path only -- the same-hardware comparator of
+ * zsm_decode_step (Sec. 4.2 compares the two end to end).  No cache handle: the caller owns K and V.
+ *   dtype      ZSM_F16 or ZSM_BF16 (UNSUPPORTED for ZSM_F32)
+ *   n_units    (layers x sequences x kv heads) handled by the call; group = query heads per kv
+ *              head (1, 2, 4, 8); head_dim 64 or 128; T tokens per unit, all attended
+ *   K, V       dev [n_units][T][head_dim];  q, out  dev [n_units][group][head_dim]
+ *   workspace  dev, 256-byte aligned, >= zsm_fullkv_workspace_bytes: per-chunk partial results
+ *              and a status word; contents need not survive between calls
+ * Asynchronous on `stream` (two kernels).  zsm_fullkv_status waits for the stream and returns
+ * the device status of the most recent call on that workspace (ZSM_ERR_TIMEOUT if a bounded
+ * wait inside the kernel gave up). */
+zsm_status_t zsm_fullkv_workspace_bytes(int32_t n_units, int32_t group, int32_t head_dim, int32_t T,
+                                        size_t *bytes);
+zsm_status_t zsm_fullkv_decode(int32_t dtype, int32_t n_units, int32_t group, int32_t head_dim,
+                               int32_t T, const void *K, const void *V, const void *q, void *out,
+                               float softmax_scale, void *workspace, size_t workspace_bytes,
+                               zsm_stream_t stream);
+zsm_status_t zsm_fullkv_status(void *workspace, zsm_stream_t stream);
+
 /* Slot capacities of unit (layer, h): token slots B_p + B_c and residual slots. */
 zsm_status_t zsm_unit_capacity(const zsm_cache_t *c, int32_t layer, int32_t h,
                                int32_t *n_token_slots, int32_t *n_residual_slots);

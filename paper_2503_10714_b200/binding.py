@@ -30,7 +30,8 @@ DTYPE_CODE = {"f32": ZSM_F32, "f16": ZSM_F16, "bf16": ZSM_BF16,
 # every symbol include/zsm.h declares
 SYMBOLS = ["zsm_split_budget", "zsm_cache_bytes", "zsm_cache_create", "zsm_cache_reset",
            "zsm_cache_free", "zsm_prefill_workspace_bytes", "zsm_prefill_compress",
-           "zsm_prefill_compress_static",
+           "zsm_prefill_compress_static", "zsm_fullkv_workspace_bytes", "zsm_fullkv_decode",
+           "zsm_fullkv_status",
            "zsm_decode_step", "zsm_decode_staging_bytes", "zsm_decode_step_host",
            "zsm_unit_capacity", "zsm_cache_export_unit", "zsm_cache_import_unit",
            "zsm_last_device_status", "zsm_decode_launch_info", "zsm_status_string"]
@@ -70,6 +71,10 @@ _lib.zsm_prefill_compress.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32,
 _lib.zsm_prefill_compress_static.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp,
                                              _vp, _vp]
 _lib.zsm_decode_step.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.zsm_fullkv_workspace_bytes.argtypes = [_i32, _i32, _i32, _i32, C.POINTER(_sz)]
+_lib.zsm_fullkv_decode.argtypes = [_i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, C.c_float, _vp,
+                                   _sz, _vp]
+_lib.zsm_fullkv_status.argtypes = [_vp, _vp]
 _lib.zsm_decode_staging_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
 _lib.zsm_decode_step_host.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.zsm_unit_capacity.argtypes = [_vp, _i32, _i32, _pi32, _pi32]
@@ -193,6 +198,28 @@ def zsm_decode_step(cache, layer, q, k_new, v_new, out, victim_pos=None, merge_s
     _check(_lib.zsm_decode_step(cache, int(layer), _dev(q), _dev(k_new), _dev(v_new), _dev(out),
                                 _dev(victim_pos), _dev(merge_slot), _stream(stream)),
            "zsm_decode_step")
+
+
+def zsm_fullkv_workspace_bytes(n_units: int, group: int, head_dim: int, T: int) -> int:
+    n = _sz()
+    _check(_lib.zsm_fullkv_workspace_bytes(int(n_units), int(group), int(head_dim), int(T),
+                                           C.byref(n)), "zsm_fullkv_workspace_bytes")
+    return n.value
+
+
+def zsm_fullkv_decode(K, V, q, out, workspace, softmax_scale=0.0, stream=None):
+    """Plain decode attention over an uncompressed cache: K, V [units, T, d]; q, out
+    [units, G, d] device tensors of one 16-bit dtype."""
+    n_units, T, d = K.shape
+    G = q.shape[1]
+    _check(_lib.zsm_fullkv_decode(int(DTYPE_CODE[K.dtype]), int(n_units), int(G), int(d), int(T),
+                                  _dev(K), _dev(V), _dev(q), _dev(out), float(softmax_scale),
+                                  _dev(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream)), "zsm_fullkv_decode")
+
+
+def zsm_fullkv_status(workspace, stream=None) -> int:
+    return int(_lib.zsm_fullkv_status(_dev(workspace), _stream(stream)))
 
 
 def zsm_decode_staging_bytes(cache, layer) -> int:

@@ -50,13 +50,6 @@ struct __align__(16) Mail {
 };
 static_assert(sizeof(Mail) == kMailFixed, "mailbox header size");
 
-template <int LANES>
-__device__ __forceinline__ float group_sum(float v) {
-#pragma unroll
-    for (int off = LANES / 2; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-    return v;
-}
-
 template <bool B>
 struct BoolC {
     static constexpr bool value = B;
@@ -102,41 +95,6 @@ __device__ __forceinline__ int treduce_index(int l) {
     return idx;
 }
 
-// G consecutive floats (one slot's weights for the whole group).
-template <int G>
-__device__ __forceinline__ void load_group(const float *p, float (&v)[G]) {
-    if constexpr (G == 1) {
-        v[0] = p[0];
-    } else if constexpr (G == 2) {
-        const float2 t = *reinterpret_cast<const float2 *>(p);
-        v[0] = t.x;
-        v[1] = t.y;
-    } else {
-#pragma unroll
-        for (int i = 0; i < G / 4; ++i) {
-            const float4 t = reinterpret_cast<const float4 *>(p)[i];
-            v[4 * i] = t.x;
-            v[4 * i + 1] = t.y;
-            v[4 * i + 2] = t.z;
-            v[4 * i + 3] = t.w;
-        }
-    }
-}
-
-template <int G>
-__device__ __forceinline__ void store_group(float *p, const float (&v)[G]) {
-    if constexpr (G == 1) {
-        p[0] = v[0];
-    } else if constexpr (G == 2) {
-        *reinterpret_cast<float2 *>(p) = make_float2(v[0], v[1]);
-    } else {
-#pragma unroll
-        for (int i = 0; i < G / 4; ++i)
-            reinterpret_cast<float4 *>(p)[i] =
-                make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    }
-}
-
 // Four consecutive elements of a row in the storage dtype, widened.
 template <typename T>
 __device__ __forceinline__ void load4(const T *p, float (&f)[4]) {
@@ -151,26 +109,6 @@ __device__ __forceinline__ void load4(const T *p, float (&f)[4]) {
         const T *e = reinterpret_cast<const T *>(&t);
 #pragma unroll
         for (int i = 0; i < 4; ++i) f[i] = Elem<T>::to_float(e[i]);
-    }
-}
-
-// One m16n8k16 tensor-core step with fp32 accumulation: c += A(16 x 16, row-major) * B(16 x 8).
-// a0..a3 and b0, b1 are packed pairs of 16-bit elements in the instruction's fragment order.
-template <typename T>
-__device__ __forceinline__ void mma_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                            uint32_t a3, uint32_t b0, uint32_t b1) {
-    if constexpr (sizeof(T) == 2 && Elem<T>::kIsBf16) {
-        asm volatile(
-            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
-            "{%8,%9}, {%0,%1,%2,%3};"
-            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-    } else {
-        asm volatile(
-            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
-            "{%8,%9}, {%0,%1,%2,%3};"
-            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
     }
 }
 
