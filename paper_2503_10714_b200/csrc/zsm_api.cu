@@ -538,6 +538,7 @@ zsm_status_t zsm_prefill_compress(zsm_cache_t *c, int32_t layer, const void *K, 
     p.W = w_eff;
     p.G = c->s.G;
     p.n_kv_heads = c->s.Hkv;
+    p.n_sm = c->n_sm;
     p.max_cap = c->layer_cap_max[layer];
     p.lambda = c->lambda;
     p.scale = c->scale;

@@ -8,9 +8,9 @@
 //   P2  the latest B_p positions are kept as they are (Sec. 3.2)
 //   P3  prefill_select     of the rest, the B_c highest (score, position) stay: radix
 //                          select of the eviction threshold, then ordered compaction
-//   P4  prefill_merge[_reg] evicted tokens, ascending position, fill-or-merge into the
+//   P4  prefill_merge[_rows] evicted tokens, ascending position, fill-or-merge into the
 //                          residual slots (Alg. 1 fill/merge branch, Eq. (hatr), (kvr));
-//                          the register form holds the merged keys in registers (B_r <= 128)
+//                          the row-per-warp form holds the merged rows in registers (B_r <= 128)
 //   P5  prefill_gather     survivors' rows, scores and positions into the unit's slots
 #include "zsm_prefill.cuh"
 
@@ -440,30 +440,36 @@ __global__ void __launch_bounds__(kMergeWarps * 32) prefill_merge_kernel(const P
 }
 
 // ---------------------------------------------------------------------------
-// P4, register form (B_r <= 32 * RT): one CTA of 256 threads per unit.  Thread (row, seg)
-// keeps D/8 consecutive floats of RT merged keys in registers (rows tid/8 + 32*j, segment
-// tid%8); merged values, which only the chosen row's threads touch, stay in shared memory.
-// Per evicted token: every thread dots its key segments with the token's, three shuffles
-// finish the dot products, a shuffle/shared-memory argmax picks the slot, the slot's eight
-// threads apply Eq. (kvr).  One barrier per token; evicted rows arrive through a cp.async
-// ring several tokens ahead.
+// P4, row-per-warp form (B_r <= 32 * RT): one CTA of 32 warps per unit.  Warp r keeps merged
+// key and value rows r, r + 32, .. in registers, D/32 elements per lane, so a dot product is
+// D/32 FMAs and five shuffles, and an update touches registers only.  Per evicted token: every
+// warp dots its rows with the token's key and posts its best (order-preserving key, slot) to
+// shared memory; one barrier; every warp reads the 32 posts with one load per lane and settles
+// the argmax with two integer warp reductions (lowest slot wins ties); the owning warp applies
+// Eq. (kvr).  A single warp issues roughly one instruction every four cycles, so the chain's
+// speed is the number of instructions on one warp's critical path: about 60 here.
+// Evicted rows arrive through a cp.async ring several tokens ahead.
 // ---------------------------------------------------------------------------
-constexpr int kRegMergeThreads = 256;
-constexpr int kRegMergePF = 10;  // ring slots; a slot is refilled two tokens after its use
-constexpr int kRegMergeIdx = (kMergeIB + kRegMergePF + 3) & ~3;  // staged positions, padded so
+constexpr int kRowMergeThreads = 1024;
+constexpr int kRowMergePF = 10;  // ring slots; a slot is refilled two tokens after its use
+constexpr int kRowMergeIdx = (kMergeIB + kRowMergePF + 3) & ~3;  // staged positions, padded so
                                                                  // the ring after them stays
                                                                  // 16-byte aligned for cp.async
 
+__device__ __forceinline__ uint32_t order_key(float f) {  // a < b  <=>  key(a) < key(b); key > 0
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
 template <typename T, int D, int RT>
-__global__ void __launch_bounds__(kRegMergeThreads) prefill_merge_reg_kernel(const PrefillParams p) {
+__global__ void __launch_bounds__(kRowMergeThreads) prefill_merge_rows_kernel(const PrefillParams p) {
     using E = Elem<T>;
     constexpr int ROWB = D * (int)sizeof(T);
     constexpr int CPR = ROWB / 16;   // 16-byte chunks per row
-    constexpr int SEG = D / 8;       // floats per thread and row
-    constexpr int PF = kRegMergePF;
-    static_assert(2 * CPR <= kRegMergeThreads, "one cp.async per thread covers a K and a V row");
-    static_assert((32 * 4 + kRegMergeIdx * 4) % 16 == 0 && (D * 4) % 16 == 0,
-                  "the ring of 16-byte copies starts on a 16-byte boundary");
+    constexpr int EPT = D / 32;      // elements of a row per lane
+    constexpr int PF = kRowMergePF;
+    static_assert(2 * CPR <= kRowMergeThreads, "one cp.async per thread covers a K and a V row");
+    static_assert((64 * 4 + kRowMergeIdx * 4) % 16 == 0, "the ring starts on a 16-byte boundary");
     extern __shared__ __align__(16) uint8_t smraw[];
 
     const int ul = blockIdx.x;
@@ -474,34 +480,32 @@ __global__ void __launch_bounds__(kRegMergeThreads) prefill_merge_reg_kernel(con
     const int32_t *evl = reinterpret_cast<const int32_t *>(p.ws + p.wl.evict_list) + (size_t)ul * T_len;
     int32_t *targets = p.dbg_targets ? p.dbg_targets + (size_t)ul * T_len : nullptr;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int seg = tid & 7, row0 = tid >> 3;
 
     if (Br == 0) {
         if (targets)
             for (int i = tid; i < n_ev; i += blockDim.x) targets[i] = -1;  // dropped (Sec. 3.2)
         return;
     }
-    float *Vr_s = reinterpret_cast<float *>(smraw);                       // [Br][D]
-    float *best_v = Vr_s + (size_t)Br * D;                                // [2][8] per-warp maxima
-    int32_t *best_r = reinterpret_cast<int32_t *>(best_v + 16);           // [2][8]
-    int32_t *idx_s = best_r + 16;                                         // [kRegMergeIdx]
-    uint8_t *ring = reinterpret_cast<uint8_t *>(idx_s + kRegMergeIdx);    // [PF][2][ROWB]
+    uint32_t *best_k = reinterpret_cast<uint32_t *>(smraw);                  // [2][32] warps' best keys
+    int32_t *best_r = reinterpret_cast<int32_t *>(best_k + 64);              // [2][32] and their slots
+    int32_t *idx_s = best_r + 64;                                            // [kRowMergeIdx]
+    uint8_t *ring = reinterpret_cast<uint8_t *>(idx_s + kRowMergeIdx);       // [PF][2][ROWB]
 
     const uint8_t *Kg = static_cast<const uint8_t *>(p.K) + (size_t)ul * T_len * ROWB;
     const uint8_t *Vg = static_cast<const uint8_t *>(p.V) + (size_t)ul * T_len * ROWB;
 
-    float kr[RT][SEG];  // this thread's segments of the merged keys
-    float wr[RT];       // their fusion counts (kept by all eight threads of a row)
+    float kr[RT][EPT], vr[RT][EPT];  // this lane's elements of the warp's merged rows
+    float wr[RT];                    // their fusion counts
 #pragma unroll
     for (int j = 0; j < RT; ++j) {
         wr[j] = 0.f;
 #pragma unroll
-        for (int e = 0; e < SEG; ++e) kr[j][e] = 0.f;
+        for (int e = 0; e < EPT; ++e) kr[j][e] = vr[j][e] = 0.f;
     }
 
     int i0 = 0;  // idx_s[j] = evl[i0 + j]
     auto stage_indices = [&](int start) {
-        for (int j = tid; j < kRegMergeIdx; j += blockDim.x)
+        for (int j = tid; j < kRowMergeIdx; j += blockDim.x)
             idx_s[j] = (start + j < n_ev) ? evl[start + j] : 0;
     };
     auto issue = [&](int i) {  // fetch evicted token i's rows into ring slot i % PF
@@ -513,15 +517,10 @@ __global__ void __launch_bounds__(kRegMergeThreads) prefill_merge_reg_kernel(con
         }
         cp_async_commit();
     };
-    auto load_seg = [&](const uint8_t *rowp, float (&f)[SEG]) {  // 16-byte loads, widened
-        const uint4 *src = reinterpret_cast<const uint4 *>(rowp + seg * SEG * sizeof(T));
+    auto load_own = [&](const uint8_t *rowp, float (&f)[EPT]) {
+        const T *src = reinterpret_cast<const T *>(rowp) + lane * EPT;
 #pragma unroll
-        for (int c = 0; c < SEG / E::EPL; ++c) {
-            float t[E::EPL];
-            E::widen(src[c], t);
-#pragma unroll
-            for (int e = 0; e < E::EPL; ++e) f[c * E::EPL + e] = t[e];
-        }
+        for (int e = 0; e < EPT; ++e) f[e] = E::to_float(src[e]);
     };
 
     stage_indices(0);
@@ -535,89 +534,73 @@ __global__ void __launch_bounds__(kRegMergeThreads) prefill_merge_reg_kernel(con
         issue(i + PF - 2);
         const uint8_t *kc_row = ring + ((size_t)(i % PF) * 2 + 0) * ROWB;
         const uint8_t *vc_row = ring + ((size_t)(i % PF) * 2 + 1) * ROWB;
-        float kc[SEG];
-        load_seg(kc_row, kc);
-        int target;
+        const int par = (i & 1) * 32;
+        float kc[EPT];
+        load_own(kc_row, kc);
+        int target = -1;
         if (i < Br) {
             target = i;  // Alg. 1: a free residual slot takes the token as it is
         } else {
-            // Eq. (hatr): raw dot products, ties to the lowest slot
-            float bv = -INFINITY;
+            // Eq. (hatr): raw dot products; within the warp ties go to the lower slot
+            float dot[RT];
+#pragma unroll
+            for (int j = 0; j < RT; ++j) {
+                float a = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) a = fmaf(kr[j][e], kc[e], a);
+                dot[j] = a;
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1)
+#pragma unroll
+                for (int j = 0; j < RT; ++j) dot[j] += __shfl_xor_sync(0xffffffffu, dot[j], off);
+            float bv = 0.f;
             int br = 0x7fffffff;
 #pragma unroll
             for (int j = 0; j < RT; ++j) {
-                float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-                for (int e = 0; e < SEG; e += 2) {
-                    a0 = fmaf(kr[j][e], kc[e], a0);
-                    a1 = fmaf(kr[j][e + 1], kc[e + 1], a1);
-                }
-                float dot = a0 + a1;
-                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-                const int r = row0 + 32 * j;
-                if (r < Br && (br == 0x7fffffff || dot > bv)) {
-                    bv = dot;
+                const int r = warp + 32 * j;
+                if (r < Br && (br == 0x7fffffff || dot[j] > bv)) {
+                    bv = dot[j];
                     br = r;
                 }
             }
-#pragma unroll
-            for (int off = 8; off <= 16; off <<= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                const int orr = __shfl_xor_sync(0xffffffffu, br, off);
-                if (orr != 0x7fffffff && (br == 0x7fffffff || ov > bv || (ov == bv && orr < br))) {
-                    bv = ov;
-                    br = orr;
-                }
-            }
             if (lane == 0) {
-                best_v[(i & 1) * 8 + warp] = bv;
-                best_r[(i & 1) * 8 + warp] = br;
+                best_k[par + warp] = br == 0x7fffffff ? 0u : order_key(bv);
+                best_r[par + warp] = br;
             }
-            target = -1;
         }
         // token i+1 must have landed before the barrier that publishes it
         cp_async_wait<PF - 3>();
         __syncthreads();
         if (target < 0) {
-            float bv = best_v[(i & 1) * 8];
-            int br = best_r[(i & 1) * 8];
-#pragma unroll
-            for (int wv = 1; wv < 8; ++wv) {
-                const float ov = best_v[(i & 1) * 8 + wv];
-                const int orr = best_r[(i & 1) * 8 + wv];
-                if (orr != 0x7fffffff && (br == 0x7fffffff || ov > bv || (ov == bv && orr < br))) {
-                    bv = ov;
-                    br = orr;
-                }
-            }
-            target = br;
+            const uint32_t key = best_k[par + lane];
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, key);
+            const int r = key == mx ? best_r[par + lane] : 0x7fffffff;
+            target = __reduce_min_sync(0xffffffffu, r);
         }
-        // Eq. (kvr) on the chosen row, by its eight threads
+        // Eq. (kvr) on the chosen row, by its warp
+        if ((target & 31) == warp) {
 #pragma unroll
-        for (int j = 0; j < RT; ++j) {
-            if (row0 + 32 * j == target) {
-                const float w = wr[j];
-                const float dn = w + 1.0f;
-                // one correctly rounded reciprocal instead of 2*SEG divisions on the chain's
-                // critical path (the divisions alone were two thirds of a merge's time)
-                const float rdn = __frcp_rn(dn);
-                float vc[SEG];
-                load_seg(vc_row, vc);
-                float *vr = Vr_s + (size_t)target * D + seg * SEG;
+            for (int j = 0; j < RT; ++j) {
+                if (warp + 32 * j == target) {
+                    const float w = wr[j];
+                    // one correctly rounded reciprocal instead of divisions on the critical path
+                    const float rdn = __frcp_rn(w + 1.0f);
+                    float vc[EPT];
+                    load_own(vc_row, vc);
 #pragma unroll
-                for (int e = 0; e < SEG; ++e) {
-                    kr[j][e] = (w == 0.f) ? kc[e] : fmaf(w, kr[j][e], kc[e]) * rdn;
-                    vr[e] = (w == 0.f) ? vc[e] : fmaf(w, vr[e], vc[e]) * rdn;
+                    for (int e = 0; e < EPT; ++e) {
+                        kr[j][e] = (w == 0.f) ? kc[e] : fmaf(w, kr[j][e], kc[e]) * rdn;
+                        vr[j][e] = (w == 0.f) ? vc[e] : fmaf(w, vr[j][e], vc[e]) * rdn;
+                    }
+                    wr[j] = w + 1.0f;
+                    if (lane == 0 && targets) targets[i] = (i < Br) ? -2 : target;
                 }
-                wr[j] = dn;
-                if (seg == 0 && targets) targets[i] = (i < Br) ? -2 : target;
             }
         }
         if (i + 1 - i0 == kMergeIB && i + 1 < n_ev) {
             // next block of positions; tokens up to i + PF - 2 were issued from the old block,
-            // whose tail (PF extra entries) covers them
+            // whose tail covers them
             __syncthreads();
             i0 = i + 1;
             stage_indices(i0);
@@ -630,23 +613,164 @@ __global__ void __launch_bounds__(kRegMergeThreads) prefill_merge_reg_kernel(con
     float *Kr_g = reinterpret_cast<float *>(p.base + d.kr_off);
     float *Vr_g = reinterpret_cast<float *>(p.base + d.vr_off);
     uint32_t *w_g = reinterpret_cast<uint32_t *>(p.base + d.w_off);
-    __syncthreads();
 #pragma unroll
     for (int j = 0; j < RT; ++j) {
-        const int r = row0 + 32 * j;
+        const int r = warp + 32 * j;
         if (r < n_res) {
 #pragma unroll
-            for (int e = 0; e < SEG; ++e) Kr_g[(size_t)r * D + seg * SEG + e] = kr[j][e];
-            if (seg == 0) w_g[r] = static_cast<uint32_t>(wr[j]);
+            for (int e = 0; e < EPT; ++e) {
+                Kr_g[(size_t)r * D + lane * EPT + e] = kr[j][e];
+                Vr_g[(size_t)r * D + lane * EPT + e] = vr[j][e];
+            }
+            if (lane == 0) w_g[r] = static_cast<uint32_t>(wr[j]);
         }
     }
-    for (int k = tid; k < n_res * D; k += blockDim.x) Vr_g[k] = Vr_s[k];
 }
 
 template <typename T, int D>
-size_t merge_reg_smem_bytes(int Br) {
-    return (size_t)Br * D * 4 + 32 * 4 + (size_t)kRegMergeIdx * 4 +
-           (size_t)kRegMergePF * 2 * D * sizeof(T);
+size_t merge_rows_smem_bytes() {
+    return (size_t)128 * 4 + (size_t)kRowMergeIdx * 4 + (size_t)kRowMergePF * 2 * D * sizeof(T);
+}
+
+// ---------------------------------------------------------------------------
+// P4, one-warp form (B_r <= 32), for layers with more units than the GPU can hold CTAs of
+// the row-per-warp form: a single warp walks a unit's chain, so a merge costs no block barrier
+// and every unit of the layer runs at once.  Lane r owns merged key r (a shared-memory row padded to D + 1 floats,
+// which makes the lanes' row-wise reads conflict-free); the token's key is widened to fp32 once,
+// cooperatively, and broadcast-read by every lane for its dot product; the argmax is one
+// integer warp reduction on order-preserving keys plus a ballot (lowest slot wins ties); the
+// chosen row and its value row are updated cooperatively, D/32 elements per lane.
+// ---------------------------------------------------------------------------
+constexpr int kWarpMergePF = 8;     // ring slots
+constexpr int kWarpMergeIB = 120;   // evicted positions staged at a time (IB + PF: multiple of 4)
+
+template <typename T, int D>
+__global__ void __launch_bounds__(32) prefill_merge_warp_kernel(const PrefillParams p) {
+    using E = Elem<T>;
+    constexpr int ROWB = D * (int)sizeof(T);
+    constexpr int CPR = ROWB / 16;
+    constexpr int EPTL = D / 32;  // elements of a row per lane in the cooperative steps
+    constexpr int LD = D + 1;     // padded key row
+    constexpr int PF = kWarpMergePF, IB = kWarpMergeIB;
+    static_assert((32 * LD * 4) % 16 == 0 && ((IB + PF) * 4) % 16 == 0, "16-byte aligned ring");
+    extern __shared__ __align__(16) uint8_t smraw[];
+
+    const int ul = blockIdx.x;
+    const UnitDesc d = p.desc[ul];
+    const int Br = d.Br;
+    const int T_len = p.T;
+    const int n_ev = reinterpret_cast<const int32_t *>(p.ws + p.wl.counts)[ul * 4];
+    const int32_t *evl = reinterpret_cast<const int32_t *>(p.ws + p.wl.evict_list) + (size_t)ul * T_len;
+    int32_t *targets = p.dbg_targets ? p.dbg_targets + (size_t)ul * T_len : nullptr;
+    const int lane = threadIdx.x;
+
+    if (Br == 0) {
+        if (targets)
+            for (int i = lane; i < n_ev; i += 32) targets[i] = -1;  // dropped (Sec. 3.2)
+        return;
+    }
+    float *Kr_s = reinterpret_cast<float *>(smraw);               // [32][LD]
+    float *Vr_s = Kr_s + 32 * LD;                                 // [32][D]
+    float *kcf = Vr_s + 32 * D;                                   // [D] the token's key, fp32
+    int32_t *idx_s = reinterpret_cast<int32_t *>(kcf + D);        // [IB + PF]
+    uint8_t *ring = reinterpret_cast<uint8_t *>(idx_s + IB + PF); // [PF][2][ROWB]
+
+    const uint8_t *Kg = static_cast<const uint8_t *>(p.K) + (size_t)ul * T_len * ROWB;
+    const uint8_t *Vg = static_cast<const uint8_t *>(p.V) + (size_t)ul * T_len * ROWB;
+
+    float wr = 0.f;  // fusion count of slot `lane`
+    int i0 = 0;
+    auto stage_indices = [&](int start) {
+        for (int j = lane; j < IB + PF; j += 32) idx_s[j] = (start + j < n_ev) ? evl[start + j] : 0;
+    };
+    auto issue = [&](int i) {
+        if (i < n_ev) {
+            const int t = idx_s[i - i0];
+            for (int c = lane; c < 2 * CPR; c += 32) {
+                const int which = c / CPR, cc = c % CPR;
+                cp_async16(ring + ((size_t)(i % PF) * 2 + which) * ROWB + cc * 16,
+                           (which ? Vg : Kg) + (size_t)t * ROWB + cc * 16);
+            }
+        }
+        cp_async_commit();
+    };
+
+    stage_indices(0);
+    __syncwarp();
+    for (int i = 0; i < PF - 1; ++i) issue(i);
+
+    for (int i = 0; i < n_ev; ++i) {
+        if (i - i0 == IB) {  // next block of positions
+            __syncwarp();
+            i0 = i;
+            stage_indices(i0);
+            __syncwarp();
+        }
+        issue(i + PF - 1);  // refills the slot of token i-1, which the warp is done with
+        cp_async_wait<PF - 1>();
+        __syncwarp();  // token i's rows are in the ring for every lane
+        const T *kc_row = reinterpret_cast<const T *>(ring + ((size_t)(i % PF) * 2 + 0) * ROWB);
+        const T *vc_row = reinterpret_cast<const T *>(ring + ((size_t)(i % PF) * 2 + 1) * ROWB);
+        float kc[EPTL], vc[EPTL];
+#pragma unroll
+        for (int e = 0; e < EPTL; ++e) {
+            kc[e] = E::to_float(kc_row[lane * EPTL + e]);
+            vc[e] = E::to_float(vc_row[lane * EPTL + e]);
+            kcf[lane * EPTL + e] = kc[e];
+        }
+        __syncwarp();
+        int target;
+        if (i < Br) {
+            target = i;  // Alg. 1: a free residual slot takes the token as it is
+        } else {
+            // Eq. (hatr): lane r's dot product of merged key r with the token's key
+            const float *kr = Kr_s + lane * LD;
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 8
+            for (int k = 0; k < D; k += 4) {
+                const float4 c4 = *reinterpret_cast<const float4 *>(kcf + k);
+                a0 = fmaf(kr[k], c4.x, a0);
+                a1 = fmaf(kr[k + 1], c4.y, a1);
+                a2 = fmaf(kr[k + 2], c4.z, a2);
+                a3 = fmaf(kr[k + 3], c4.w, a3);
+            }
+            const float dot = (a0 + a1) + (a2 + a3);
+            const uint32_t key = lane < Br ? order_key(dot) : 0u;
+            const uint32_t best = __reduce_max_sync(0xffffffffu, key);
+            target = __ffs(__ballot_sync(0xffffffffu, key == best && lane < Br)) - 1;
+        }
+        // Eq. (kvr) on the chosen row, D/32 elements per lane
+        const float w = __shfl_sync(0xffffffffu, wr, target);
+        const float rdn = __frcp_rn(w + 1.0f);
+        float *krow = Kr_s + target * LD + lane * EPTL;
+        float *vrow = Vr_s + target * D + lane * EPTL;
+#pragma unroll
+        for (int e = 0; e < EPTL; ++e) {
+            krow[e] = (w == 0.f) ? kc[e] : fmaf(w, krow[e], kc[e]) * rdn;
+            vrow[e] = (w == 0.f) ? vc[e] : fmaf(w, vrow[e], vc[e]) * rdn;
+        }
+        if (lane == target) wr = w + 1.0f;
+        if (lane == 0 && targets) targets[i] = (i < Br) ? -2 : target;
+        __syncwarp();  // the updated row is in place before the next token's dot products
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+
+    const int n_res = min(Br, n_ev);
+    float *Kr_g = reinterpret_cast<float *>(p.base + d.kr_off);
+    float *Vr_g = reinterpret_cast<float *>(p.base + d.vr_off);
+    uint32_t *w_g = reinterpret_cast<uint32_t *>(p.base + d.w_off);
+    for (int k = lane; k < n_res * D; k += 32) {
+        Kr_g[k] = Kr_s[(k / D) * LD + (k % D)];
+        Vr_g[k] = Vr_s[k];
+    }
+    if (lane < n_res) w_g[lane] = static_cast<uint32_t>(wr);
+}
+
+template <typename T, int D>
+size_t merge_warp_smem_bytes() {
+    return (size_t)32 * (D + 1) * 4 + (size_t)32 * D * 4 + (size_t)D * 4 +
+           (size_t)(kWarpMergeIB + kWarpMergePF) * 4 + (size_t)kWarpMergePF * 2 * D * sizeof(T);
 }
 
 // ---------------------------------------------------------------------------
@@ -709,13 +833,16 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
         scores = reinterpret_cast<const float *>(p.ws + p.wl.scores);
     }
     prefill_select_kernel<<<p.units, 1024, 0, stream>>>(p, scores);
-    // the residual chain: merged keys in registers when the layer's largest B_r allows it
-    if (max_br <= 32)
-        prefill_merge_reg_kernel<T, D, 1><<<p.units, kRegMergeThreads, merge_reg_smem_bytes<T, D>(max_br), stream>>>(p);
+    // the residual chain: merged rows in registers, one per warp, up to 128 merged slots (one
+    // warp per unit when the layer has many units); the shared-memory form beyond
+    if (max_br <= 32 && p.units > 2 * p.n_sm)  // more chains than row-per-warp CTAs fit at once
+        prefill_merge_warp_kernel<T, D><<<p.units, 32, merge_warp_smem_bytes<T, D>(), stream>>>(p);
+    else if (max_br <= 32)
+        prefill_merge_rows_kernel<T, D, 1><<<p.units, kRowMergeThreads, merge_rows_smem_bytes<T, D>(), stream>>>(p);
     else if (max_br <= 64)
-        prefill_merge_reg_kernel<T, D, 2><<<p.units, kRegMergeThreads, merge_reg_smem_bytes<T, D>(max_br), stream>>>(p);
+        prefill_merge_rows_kernel<T, D, 2><<<p.units, kRowMergeThreads, merge_rows_smem_bytes<T, D>(), stream>>>(p);
     else if (max_br <= 128)
-        prefill_merge_reg_kernel<T, D, 4><<<p.units, kRegMergeThreads, merge_reg_smem_bytes<T, D>(max_br), stream>>>(p);
+        prefill_merge_rows_kernel<T, D, 4><<<p.units, kRowMergeThreads, merge_rows_smem_bytes<T, D>(), stream>>>(p);
     else
         prefill_merge_kernel<T, D><<<p.units, kMergeWarps * 32,
                                      merge_smem_bytes<D>(max_br, D * (int)sizeof(T)), stream>>>(p);
@@ -735,14 +862,8 @@ int prepare_all() {
                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)merge_smem_bytes<D>(prefill_max_residual(D), D * (int)sizeof(T)));
     if (e != cudaSuccess) return static_cast<int>(e);
-    e = cudaFuncSetAttribute(prefill_merge_reg_kernel<T, D, 1>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_reg_smem_bytes<T, D>(32));
-    if (e != cudaSuccess) return static_cast<int>(e);
-    e = cudaFuncSetAttribute(prefill_merge_reg_kernel<T, D, 2>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_reg_smem_bytes<T, D>(64));
-    if (e != cudaSuccess) return static_cast<int>(e);
-    e = cudaFuncSetAttribute(prefill_merge_reg_kernel<T, D, 4>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_reg_smem_bytes<T, D>(128));
+    e = cudaFuncSetAttribute(prefill_merge_warp_kernel<T, D>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_warp_smem_bytes<T, D>());
     return static_cast<int>(e);
 }
 

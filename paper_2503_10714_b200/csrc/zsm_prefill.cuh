@@ -55,6 +55,7 @@ struct PrefillParams {
     uint8_t *dbg_evicted;      // [units][T] or null
     int32_t *dbg_targets;      // [units][T] or null
     int32_t units, T, W, G, n_kv_heads;
+    int32_t n_sm;              // SMs of the device (picks the form of the merge kernel)
     int32_t max_cap;           // largest B_p + B_c among these units
     float lambda, scale;
 };

@@ -95,6 +95,19 @@ def test_residual_pool_sizes(zb, oracle, br):
         cache.close()
 
 
+def test_layer_with_more_units_than_resident_ctas(zb, oracle):
+    """320 units in one layer: more chains than the GPU holds CTAs of the row-per-warp merge
+    kernel, so the one-warp form runs; every unit is checked."""
+    w = wl.Workload("many", 1, 40, 8, 8, 64, "bf16", 260, 0, 8, None, 26)
+    cache = GpuCache(zb, w, np.full((1, 8), 12), np.full((1, 8), 20), np.arange(1, 9).reshape(1, 8) * 4)
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats)
+        assert cache.status() == 0 and stats.merges > 40000
+    finally:
+        cache.close()
+
+
 def test_supplied_scores_with_exact_ties(zb, oracle):
     """Scores given by the caller, drawn from four values only: the selection is decided by
     the position rule almost everywhere and must match the oracle bit for bit (no near tie
