@@ -20,3 +20,15 @@ def test_merging_beats_eviction_at_every_ratio():
     ratios = sorted(res, reverse=True)
     for a, b in zip(ratios, ratios[1:]):
         assert res[a]["evict"] < res[b]["evict"] and res[a]["merge"] < res[b]["merge"]
+
+
+def test_compensation_term_is_what_makes_merging_pay():
+    """Sensitivity axis alpha (App. C.2 / Sec. 3.5): with alpha = 0 a merged slot weighs like one
+    token and the output error is close to eviction's; alpha = 1 cuts it several-fold."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2503_10714_b200 import error_analysis
+    kw = dict(ratios=(0.1,), prompt_len=2048, steps=48)
+    e1 = error_analysis.run(alpha=1.0, **kw)[0.1]
+    e0 = error_analysis.run(alpha=0.0, **kw)[0.1]
+    assert e1["merge"] < 0.6 * e0["merge"] and e0["merge"] > 0.8 * e0["evict"]
