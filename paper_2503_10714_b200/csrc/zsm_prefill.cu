@@ -2,7 +2,8 @@
 //
 //   P1  scores from the prompt's last W queries: causal softmax rows combined by
 //       Eq. (score) unrolled, s_t = (1/G) sum_g sum_tau lambda^(T-1-tau) a_t^(tau)
-//         prefill_logits   scaled, masked q.k into scratch + per-chunk (max, sum exp)
+//         prefill_logits[_mma]  scaled, masked q.k into scratch + per-chunk (max, sum exp);
+//                          16-bit storage: on the tensor cores
 //         prefill_rowstat  per query row: max and weight/sum
 //         prefill_scores   s_t = sum_rows exp(logit - max) * weight/sum
 //   P2  the latest B_p positions are kept as they are (Sec. 3.2)
@@ -128,6 +129,124 @@ __global__ void __launch_bounds__(256) prefill_logits_kernel(const PrefillParams
             if (tx == 0) partial[(size_t)gw * n_chunks + blockIdx.x] = make_float2(m, sum);
         }
     }
+}
+
+// ---------------------------------------------------------------------------
+// P1a on the tensor cores (16-bit storage): the window scoring is a dense
+// (G*W) x d x T contraction, 32 flop per K byte at G*W = 32 -- above what plain
+// FMAs can do at HBM speed.  Same grid and outputs as prefill_logits_kernel.
+// Warp w owns positions 16w .. 16w+15 of the chunk: their A fragments are read once
+// (mma.sync m16n8k16, contraction index permuted as in the decode kernel) and reused
+// for every block of eight query rows.  Scaled, masked logits go through a shared
+// tile, which gives coalesced row writes and the per-row (max, sum exp) of the chunk.
+// ---------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(256) prefill_logits_mma_kernel(const PrefillParams p) {
+    static_assert(sizeof(T) == 2, "16-bit storage");
+    constexpr int CH = kPrefillChunk;  // 128 positions = 8 warps x 16 rows
+    constexpr int ROWB = D * 2;
+    constexpr int SEG = ROWB / 64;
+    constexpr int LT = CH + 4;         // padded tile row (floats)
+    extern __shared__ __align__(16) uint8_t smb[];
+    uint8_t *Ks = smb;                                   // [CH][ROWB]   keys of the chunk
+    uint8_t *Qs = Ks + CH * ROWB;                        // [kQB][ROWB]  current block of queries
+    float *lt = reinterpret_cast<float *>(Qs + kQB * ROWB);  // [kQB][LT] logits of the block
+
+    const int ul = blockIdx.y;
+    const int b = ul / p.n_kv_heads, h = ul % p.n_kv_heads;
+    const int t0 = blockIdx.x * CH;
+    const int T_len = p.T, W = p.W, G = p.G, GW = p.G * p.W;
+    const int n_chunks = gridDim.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gq = lane >> 2, tig = lane & 3;
+    const uint8_t *Kg = static_cast<const uint8_t *>(p.K) + ((size_t)ul * T_len) * ROWB;
+    const int n_q_heads = p.n_kv_heads * G;
+
+    for (int k = tid; k < CH * (ROWB / 16); k += 256) {
+        const int r = k / (ROWB / 16), c = k % (ROWB / 16);
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (t0 + r < T_len) v = *reinterpret_cast<const uint4 *>(Kg + (size_t)(t0 + r) * ROWB + c * 16);
+        *reinterpret_cast<uint4 *>(Ks + r * ROWB + c * 16) = v;
+    }
+    __syncthreads();
+    // this warp's 16 positions as A fragments, all segments
+    uint4 fa[SEG], fc[SEG];
+    {
+        const uint8_t *pa = Ks + (warp * 16 + gq) * ROWB + tig * 16;
+#pragma unroll
+        for (int j = 0; j < SEG; ++j) {
+            fa[j] = *reinterpret_cast<const uint4 *>(pa + j * 64);
+            fc[j] = *reinterpret_cast<const uint4 *>(pa + 8 * ROWB + j * 64);
+        }
+    }
+    float *logits = reinterpret_cast<float *>(p.ws + p.wl.logits) + (size_t)ul * GW * T_len;
+    float2 *partial = reinterpret_cast<float2 *>(p.ws + p.wl.partial) + (size_t)ul * GW * n_chunks;
+
+    for (int qb = 0; qb < GW; qb += kQB) {
+        __syncthreads();  // the previous block's tile and queries are no longer read
+        for (int k = tid; k < kQB * (ROWB / 16); k += 256) {
+            const int r = k / (ROWB / 16), c = k % (ROWB / 16);
+            const int gw = qb + r;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (gw < GW) {
+                const int g = gw / W, wq = gw % W;
+                v = *reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(p.Qw) +
+                        (((size_t)b * n_q_heads + h * G + g) * W + wq) * ROWB + c * 16);
+            }
+            *reinterpret_cast<uint4 *>(Qs + r * ROWB + c * 16) = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int nb = 0; nb < kQB / 8; ++nb) {
+            float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint8_t *pq = Qs + (nb * 8 + gq) * ROWB + tig * 16;
+#pragma unroll
+            for (int j = 0; j < SEG; ++j) {
+                const uint4 qv = *reinterpret_cast<const uint4 *>(pq + j * 64);
+                mma_16x8x16<T>(c0, fa[j].x, fc[j].x, fa[j].y, fc[j].y, qv.x, qv.y);
+                mma_16x8x16<T>(c1, fa[j].z, fc[j].z, fa[j].w, fc[j].w, qv.z, qv.w);
+            }
+            // rows gq, gq+8 of the warp's positions; query rows nb*8 + tig*2, +1
+            const int pos = warp * 16 + gq;
+            const int qr = nb * 8 + tig * 2;
+            lt[qr * LT + pos] = (c0[0] + c1[0]) * p.scale;
+            lt[(qr + 1) * LT + pos] = (c0[1] + c1[1]) * p.scale;
+            lt[qr * LT + pos + 8] = (c0[2] + c1[2]) * p.scale;
+            lt[(qr + 1) * LT + pos + 8] = (c0[3] + c1[3]) * p.scale;
+        }
+        __syncthreads();
+        // warp w: query rows 4w .. 4w+3 of the block; lane: positions lane + 32 i
+#pragma unroll
+        for (int jr = 0; jr < 4; ++jr) {
+            const int gw = qb + warp * 4 + jr;
+            if (gw >= GW) continue;  // uniform per warp
+            const int tau = T_len - W + (gw % W);  // the query's own position: keys 0..tau
+            float m = -INFINITY;
+            float lg[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int t = t0 + lane + 32 * i;
+                lg[i] = (t < T_len && t <= tau) ? lt[(warp * 4 + jr) * LT + lane + 32 * i] : -INFINITY;
+                if (t < T_len) logits[(size_t)gw * T_len + t] = lg[i];
+                m = fmaxf(m, lg[i]);
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+            float sum = 0.f;
+            if (m > -INFINITY) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sum += expf(lg[i] - m);
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+            if (lane == 0) partial[(size_t)gw * n_chunks + blockIdx.x] = make_float2(m, sum);
+        }
+    }
+}
+
+template <int D>
+size_t logits_mma_smem_bytes() {
+    return (size_t)(kPrefillChunk + kQB) * D * 2 + (size_t)kQB * (kPrefillChunk + 4) * 4;
 }
 
 // P1b: one thread per (unit, query row): fold the chunk partials.
@@ -826,7 +945,10 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
     const float *scores = p.scores_in;
     if (p.Qw) {
         const size_t sm = (size_t)(kPrefillChunk + kQB) * (D + 4) * 4;
-        prefill_logits_kernel<T, D><<<dim3(n_chunks, p.units), 256, sm, stream>>>(p);
+        if constexpr (sizeof(T) == 2)
+            prefill_logits_mma_kernel<T, D><<<dim3(n_chunks, p.units), 256, logits_mma_smem_bytes<D>(), stream>>>(p);
+        else
+            prefill_logits_kernel<T, D><<<dim3(n_chunks, p.units), 256, sm, stream>>>(p);
         const int rows = p.units * p.G * p.W;
         prefill_rowstat_kernel<<<(rows + 127) / 128, 128, 0, stream>>>(p, n_chunks);
         prefill_scores_kernel<<<dim3((p.T + 255) / 256, p.units), 256, 0, stream>>>(p);
@@ -854,6 +976,12 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
 
 template <typename T, int D>
 int prepare_all() {
+    if constexpr (sizeof(T) == 2) {
+        cudaError_t e2 = cudaFuncSetAttribute(prefill_logits_mma_kernel<T, D>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)logits_mma_smem_bytes<D>());
+        if (e2 != cudaSuccess) return static_cast<int>(e2);
+    }
     cudaError_t e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)((kPrefillChunk + kQB) * (D + 4) * 4));
