@@ -82,8 +82,10 @@ typedef struct {
     float softmax_scale; /* 0 selects 1/sqrt(head_dim) [Eq. (att_score)] */
     /* Launch tuning of the fused decode kernel; 0 selects the library default. */
     int32_t tune_stages;         /* 16 KiB ring stages per CTA */
-    int32_t tune_ctas_per_sm;    /* persistent CTAs per SM (default 2) */
-    int32_t tune_consumer_warps; /* compute warps per CTA, at most 8 (two more warps feed them
+    int32_t tune_ctas_per_sm;    /* persistent CTAs per SM (default: 2, or 1 for a launch with no
+                                  * more units than SMs) */
+    int32_t tune_consumer_warps; /* compute warps per CTA: at most 8 with two CTAs per SM, 16 with
+                                  * one (two more warps feed them
                                   * and write the cache update back) */
 } zsm_config_t;
 

@@ -45,8 +45,14 @@ struct zsm_cache {
     uint8_t *base;
     size_t bytes;
     Layout lay;
-    int n_sm, stages, ctas_per_sm, consumer_warps;
-    int grid_all, grid_layer;
+    int n_sm;
+    // Launch plan of the fused decode kernel, one for the all-layer launch and one for a
+    // single layer's: a launch with no more units than SMs runs the wide form (one CTA per SM,
+    // sixteen consumer warps, the whole shared memory as ring), otherwise two CTAs per SM.
+    struct Plan {
+        int ctas_per_sm, consumer_warps, stages, smem_bytes, grid;
+        bool wide;
+    } plan_all, plan_layer;
     int l_stride, br_max, br_max_pad, cap_max;
     int smem_bytes;
     std::vector<int> layer_cap_max, layer_br_max;
@@ -313,46 +319,58 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
     c->br_max_pad = (c->br_max + 3) & ~3;
     c->l_stride = (ent_max + 3) & ~3;
 
-    // ---- launch plan of the fused decode kernel ----
-    // Two CTAs per SM by default: one CTA's per-unit serial phases (softmax reductions, victim
-    // search, merge) overlap the other's streaming.
-    c->ctas_per_sm = cfg->tune_ctas_per_sm > 0 ? cfg->tune_ctas_per_sm : 2;
-    c->consumer_warps = cfg->tune_consumer_warps > 0 ? cfg->tune_consumer_warps : 8;
-    if (c->consumer_warps > kMaxConsumerWarps || c->ctas_per_sm > 8) {
-        delete c;
-        return ZSM_ERR_INVALID_ARG;
-    }
-    const int header_bytes =
-        16 + (int)sizeof(UnitDesc) + (s.G + 2) * s.row_bytes + c->br_max_pad * 4;
-    const int per_cta_budget = kMaxSmemPerCta / c->ctas_per_sm - 1024 * (c->ctas_per_sm > 1);
-    const int fixed = decode_smem_total(c, 0, c->consumer_warps);
-    int stages = (per_cta_budget - fixed - 64) / (kTileBytes + 16);
-    if (cfg->tune_stages > 0) stages = std::min(stages, (int)cfg->tune_stages);
-    stages = std::min(stages, 12);
-    while (stages >= 2 && decode_smem_total(c, stages, c->consumer_warps) > per_cta_budget) --stages;
-    if (header_bytes > kTileBytes || stages < 2) {
-        delete c;
-        return ZSM_ERR_UNSUPPORTED;  // budget too large for the shared-memory weight array
-    }
-    c->stages = stages;
-    c->smem_bytes = decode_smem_total(c, stages, c->consumer_warps);
+    // ---- launch plans of the fused decode kernel ----
     if (c->br_max > prefill_max_residual(s.D)) {
         delete c;
         return ZSM_ERR_UNSUPPORTED;
     }
-    int occ = 0;
-    int rc = prepare_decode_fused(s.dtype, s.D, s.G, c->smem_bytes, (c->consumer_warps + kExtraWarps) * 32, &occ);
-    if (rc != 0 || prepare_prefill(s.dtype, s.D) != 0) {
+    if (prepare_prefill(s.dtype, s.D) != 0) {
         delete c;
-        return rc == -1 ? ZSM_ERR_UNSUPPORTED : ZSM_ERR_CUDA;
+        return ZSM_ERR_CUDA;
     }
-    if (occ < 1) {
+    const int header_bytes =
+        16 + (int)sizeof(UnitDesc) + (s.G + 2) * s.row_bytes + c->br_max_pad * 4;
+    if (header_bytes > kTileBytes) {
         delete c;
         return ZSM_ERR_UNSUPPORTED;
     }
-    c->ctas_per_sm = std::min(c->ctas_per_sm, occ);
-    c->grid_all = std::min(default_grid(s.n_units, c->n_sm, c->ctas_per_sm), 1024);
-    c->grid_layer = std::min(default_grid(s.upl, c->n_sm, c->ctas_per_sm), 1024);
+    auto make_plan = [&](int units, zsm_cache::Plan &pl) -> zsm_status_t {
+        const bool solo = units <= c->n_sm;  // a CTA has an SM to itself whatever we do
+        pl.ctas_per_sm = cfg->tune_ctas_per_sm > 0 ? cfg->tune_ctas_per_sm : (solo ? 1 : 2);
+        pl.consumer_warps = cfg->tune_consumer_warps > 0
+                                ? cfg->tune_consumer_warps
+                                : (pl.ctas_per_sm == 1 ? kMaxConsumerWarps : kPairConsumerWarps);
+        pl.wide = pl.ctas_per_sm == 1;
+        if (pl.ctas_per_sm > 8 || pl.consumer_warps > (pl.wide ? kMaxConsumerWarps : kPairConsumerWarps))
+            return ZSM_ERR_INVALID_ARG;
+        const int budget = kMaxSmemPerCta / pl.ctas_per_sm - 1024 * (pl.ctas_per_sm > 1);
+        const int fixed = decode_smem_total(c, 0, pl.consumer_warps);
+        int stages = (budget - fixed - 64) / (kTileBytes + 16);
+        if (cfg->tune_stages > 0) stages = std::min(stages, (int)cfg->tune_stages);
+        stages = std::min(stages, 12);
+        while (stages >= 2 && decode_smem_total(c, stages, pl.consumer_warps) > budget) --stages;
+        if (stages < 2) return ZSM_ERR_UNSUPPORTED;  // budget too large for the weight array
+        pl.stages = stages;
+        pl.smem_bytes = decode_smem_total(c, stages, pl.consumer_warps);
+        int occ = 0;
+        const int rc = prepare_decode_fused(s.dtype, s.D, s.G, pl.smem_bytes,
+                                            (pl.consumer_warps + kExtraWarps) * 32, &occ);
+        if (rc != 0) return rc == -1 ? ZSM_ERR_UNSUPPORTED : ZSM_ERR_CUDA;
+        if (!pl.wide) {
+            if (occ < 1) return ZSM_ERR_UNSUPPORTED;
+            pl.ctas_per_sm = std::min(pl.ctas_per_sm, occ);
+        }
+        pl.grid = std::min(default_grid(units, c->n_sm, pl.ctas_per_sm), 1024);
+        return ZSM_OK;
+    };
+    {
+        zsm_status_t ps = make_plan(s.n_units, c->plan_all);
+        if (ps == ZSM_OK) ps = make_plan(s.upl, c->plan_layer);
+        if (ps != ZSM_OK) {
+            delete c;
+            return ps;
+        }
+    }
 
     // same table sizes as zsm_cache_bytes, so the byte count never depends on the device
     build_layout(s, c->Bp.data(), c->Bc.data(), c->Br.data(), std::min(s.n_units, 1024),
@@ -367,7 +385,7 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
     std::vector<UnitDesc> dl;
     units.resize(s.n_units);
     for (int u = 0; u < s.n_units; ++u) units[u] = u;
-    lpt_schedule(units, lay.desc, s.row_bytes, s.D, c->grid_all, off, order);
+    lpt_schedule(units, lay.desc, s.row_bytes, s.D, c->plan_all.grid, off, order);
     dl.resize(order.size());
     for (size_t i = 0; i < order.size(); ++i) dl[i] = lay.desc[order[i]];
     put(lay.sched_all_off, off.data(), off.size() * 4);
@@ -375,7 +393,7 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
     for (int l = 0; l < s.L; ++l) {
         units.resize(s.upl);
         for (int u = 0; u < s.upl; ++u) units[u] = l * s.upl + u;
-        lpt_schedule(units, lay.desc, s.row_bytes, s.D, c->grid_layer, off, order);
+        lpt_schedule(units, lay.desc, s.row_bytes, s.D, c->plan_layer.grid, off, order);
         dl.resize(order.size());
         for (size_t i = 0; i < order.size(); ++i) dl[i] = lay.desc[order[i]];
         put(lay.sched_layer_off[l], off.data(), off.size() * 4);
@@ -418,9 +436,10 @@ zsm_status_t zsm_unit_capacity(const zsm_cache_t *c, int32_t layer, int32_t h,
 zsm_status_t zsm_decode_launch_info(const zsm_cache_t *c, int32_t layer, int32_t *grid,
                                     int32_t *block, int32_t *dynamic_smem_bytes) {
     if (!c || layer < -1 || layer >= c->s.L) return ZSM_ERR_INVALID_ARG;
-    if (grid) *grid = layer < 0 ? c->grid_all : c->grid_layer;
-    if (block) *block = (c->consumer_warps + kExtraWarps) * 32;
-    if (dynamic_smem_bytes) *dynamic_smem_bytes = c->smem_bytes;
+    const zsm_cache::Plan &pl = layer < 0 ? c->plan_all : c->plan_layer;
+    if (grid) *grid = pl.grid;
+    if (block) *block = (pl.consumer_warps + kExtraWarps) * 32;
+    if (dynamic_smem_bytes) *dynamic_smem_bytes = pl.smem_bytes;
     return ZSM_OK;
 }
 
@@ -451,15 +470,15 @@ zsm_status_t zsm_decode_step(zsm_cache_t *c, int32_t layer, const void *q, const
     p.out = out;
     p.victim_pos = victim_pos;
     p.merge_slot = merge_slot;
-    p.stages = c->stages;
+    const zsm_cache::Plan &pl = layer < 0 ? c->plan_all : c->plan_layer;
+    p.stages = pl.stages;
     p.l_stride = c->l_stride;
     p.br_max_pad = c->br_max_pad;
     p.lambda = c->lambda;
     p.alpha = c->alpha;
     p.scale = c->scale;
-    const int grid = layer < 0 ? c->grid_all : c->grid_layer;
-    const int rc = launch_decode_fused(c->s.dtype, c->s.D, c->s.G, p, grid, c->consumer_warps,
-                                       static_cast<cudaStream_t>(stream));
+    const int rc = launch_decode_fused(c->s.dtype, c->s.D, c->s.G, p, pl.grid, pl.consumer_warps,
+                                       pl.wide, static_cast<cudaStream_t>(stream));
     if (rc == -1) return ZSM_ERR_UNSUPPORTED;
     return rc == 0 ? ZSM_OK : ZSM_ERR_CUDA;
 }

@@ -29,7 +29,8 @@ namespace zsm {
 
 namespace {
 
-constexpr int kMaxThreads = (kMaxConsumerWarps + kExtraWarps) * 32;
+constexpr int kMaxThreads = (kMaxConsumerWarps + kExtraWarps) * 32;    // wide form, one CTA per SM
+constexpr int kPairThreads = (kPairConsumerWarps + kExtraWarps) * 32;  // two CTAs per SM
 constexpr int kMaxDynamicSmem = 232448;  // 227 KiB, the opt-in limit per CTA on sm_100
 
 // "where" codes recorded with a timeout
@@ -112,8 +113,12 @@ __device__ __forceinline__ void load4(const T *p, float (&f)[4]) {
     }
 }
 
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const DecodeParams p) {
+// WIDE: up to sixteen consumer warps in one CTA per SM, for launches with no more units than
+// SMs, where a CTA has an SM to itself and its speed is what its warps can consume; otherwise
+// up to eight consumer warps and two CTAs per SM.  Same code: the warp count is the launch's.
+template <typename T, int D, int G, bool WIDE>
+__global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 2)
+    decode_fused_kernel(const DecodeParams p) {
     using E = Elem<T>;
     constexpr int EPL = E::EPL;               // elements per 16-byte lane load
     constexpr int EP2 = EPL / 2;
@@ -464,9 +469,14 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
     };
     auto csync = [&]() { named_bar_sync(1, NT); };
 
-    // a full tile needs no row checks when the warps' row groups tile it exactly
-    const bool full_k = (R % (NW * RPW * UBK)) == 0;
-    const bool full_v = (R % (NW * RPW * UBV)) == 0;
+    // A tile's rows are shared by a group of warps, kg (logits, FMA form) or vg (output) of
+    // them; when there are more consumer warps than that, the groups take tiles in turn.
+    const int kg = max(1, min(NW, R / (RPW * UBK)));
+    const int vg = max(1, min(NW, R / (RPW * UBV)));
+    const int n_kgroups = NW / kg, n_vgroups = NW / vg;
+    // a full tile needs no row checks when the group's row sets tile it exactly
+    const bool full_k = (R % (kg * RPW * UBK)) == 0;
+    const bool full_v = (R % (vg * RPW * UBV)) == 0;
     const int rb_step = RB % NW;  // how far a tile's 16-row blocks advance the round-robin
     // where this lane's sums land after the transposing reduction of the logits pass
     const int tr_idx = treduce_index<NV, LPR>(l);
@@ -543,7 +553,7 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
         release();
 
         // ---------------- D1: logits of the token slots ----------------
-        int kturn = 0;
+        int kturn = 0, gturn = 0;
         for (int r0 = 0; r0 < n_live; r0 += R) {
             const uint8_t *tile = wait_full(W_K);
             if (!tile) return;
@@ -582,13 +592,14 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
                 kturn += rb_step;
                 if (kturn >= NW) kturn -= NW;
             } else {
+                const int wk = warp - gturn * kg;  // this warp's place in the tile's group
                 auto k_rows = [&](auto full) {
                     constexpr bool FULL = decltype(full)::value;  // every row of the pass exists
-                    for (int base = warp * RPW; base < rows; base += NW * RPW * UBK) {
+                    for (int base = wk * RPW; base < rows; base += kg * RPW * UBK) {
                         uint4 raw[UBK];
     #pragma unroll
                         for (int u = 0; u < UBK; ++u) {
-                            const int row = base + u * NW * RPW + sub;
+                            const int row = base + u * kg * RPW + sub;
                             raw[u] = (FULL || row < rows)
                                          ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
                                          : make_uint4(0, 0, 0, 0);
@@ -613,13 +624,16 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
                             for (int k = 0; k < NF; ++k) {
                                 const int id = tr_idx + k;
                                 const int u = id / G, g = id % G;
-                                const int row = base + u * NW * RPW + sub;
+                                const int row = base + u * kg * RPW + sub;
                                 if (FULL || row < rows) probs[(r0 + row) * G + g] = v[k] * p.scale;
                             }
                         }
                     }
                 };
-                if (rows == R && full_k) k_rows(BoolC<true>{}); else k_rows(BoolC<false>{});
+                if (wk >= 0 && wk < kg) {
+                    if (rows == R && full_k) k_rows(BoolC<true>{}); else k_rows(BoolC<false>{});
+                }
+                if (++gturn == n_kgroups) gturn = 0;
             }
             release();
         }
@@ -816,24 +830,26 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
         for (int g = 0; g < G; ++g)
 #pragma unroll
             for (int e = 0; e < EP2; ++e) acc2[g][e] = make_float2(0.f, 0.f);
+        int vturn = 0;
         for (int r0 = 0; r0 < n_live; r0 += R) {
             const uint8_t *tile = wait_full(W_V);
             if (!tile) return;
             const int rows = min(R, n_live - r0);
+            const int wv_ = warp - vturn * vg;  // this warp's place in the tile's group
             auto v_rows = [&](auto full) {
                 constexpr bool FULL = decltype(full)::value;
-                for (int base = warp * RPW; base < rows; base += NW * RPW * UBV) {
+                for (int base = wv_ * RPW; base < rows; base += vg * RPW * UBV) {
                     uint4 raw[UBV];
 #pragma unroll
                     for (int u = 0; u < UBV; ++u) {
-                        const int row = base + u * NW * RPW + sub;
+                        const int row = base + u * vg * RPW + sub;
                         raw[u] = (FULL || row < rows)
                                      ? *reinterpret_cast<const uint4 *>(tile + row * ROWB + l * 16)
                                      : make_uint4(0, 0, 0, 0);
                     }
 #pragma unroll
                     for (int u = 0; u < UBV; ++u) {
-                        const int row = base + u * NW * RPW + sub;
+                        const int row = base + u * vg * RPW + sub;
                         float f[EPL];
                         E::widen(raw[u], f);
                         float pv[G];
@@ -853,7 +869,10 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
                     }
                 }
             };
-            if (rows == R && full_v) v_rows(BoolC<true>{}); else v_rows(BoolC<false>{});
+            if (wv_ >= 0 && wv_ < vg) {
+                if (rows == R && full_v) v_rows(BoolC<true>{}); else v_rows(BoolC<false>{});
+            }
+            if (++vturn == n_vgroups) vturn = 0;
             release();
         }
         float acc32[G][4];
@@ -925,24 +944,31 @@ __global__ void __launch_bounds__(kMaxThreads, 2) decode_fused_kernel(const Deco
 }
 
 template <typename T, int D, int G>
-int launch_one(const DecodeParams &p, int grid, int consumer_warps, cudaStream_t stream) {
+int launch_one(const DecodeParams &p, int grid, int consumer_warps, bool wide, cudaStream_t stream) {
     const int threads = (consumer_warps + kExtraWarps) * 32;
     const DecodeSmem L = decode_smem_layout(p.stages, G, D, D * (int)sizeof(T), p.l_stride,
                                             p.br_max_pad, consumer_warps);
-    decode_fused_kernel<T, D, G><<<grid, threads, L.total, stream>>>(p);
+    if (wide)
+        decode_fused_kernel<T, D, G, true><<<grid, threads, L.total, stream>>>(p);
+    else
+        decode_fused_kernel<T, D, G, false><<<grid, threads, L.total, stream>>>(p);
     return static_cast<int>(cudaGetLastError());
 }
 
 template <typename T, int D, int G>
 int prepare_one(int smem_bytes, int threads, int *max_ctas) {
+    cudaError_t ew = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, true>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          kMaxDynamicSmem);
+    if (ew != cudaSuccess) return static_cast<int>(ew);
     // The limit belongs to the kernel, not to a cache: caches of one shape but different budgets
     // ask for different amounts, so it is raised to the most any of them can ask for.
-    cudaError_t e = cudaFuncSetAttribute(decode_fused_kernel<T, D, G>,
+    cudaError_t e = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kMaxDynamicSmem);
     if (e != cudaSuccess) return static_cast<int>(e);
     int n = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_fused_kernel<T, D, G>, threads,
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_fused_kernel<T, D, G, false>, threads,
                                                       smem_bytes);
     if (max_ctas) *max_ctas = n;
     return static_cast<int>(e);
@@ -973,8 +999,8 @@ int prepare_one(int smem_bytes, int threads, int *max_ctas) {
 }  // namespace
 
 int launch_decode_fused(int dtype, int D, int G, const DecodeParams &p, int grid,
-                        int consumer_warps, cudaStream_t stream) {
-    ZSM_DISPATCH(launch_one, p, grid, consumer_warps, stream);
+                        int consumer_warps, bool wide, cudaStream_t stream) {
+    ZSM_DISPATCH(launch_one, p, grid, consumer_warps, wide, stream);
     return -1;
 }
 

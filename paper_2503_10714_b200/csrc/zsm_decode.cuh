@@ -6,7 +6,8 @@
 namespace zsm {
 
 constexpr int kTileBytes = 16384;     // one ring stage
-constexpr int kMaxConsumerWarps = 8;  // + 1 producer warp + 1 tail warp
+constexpr int kMaxConsumerWarps = 16;  // wide form (one CTA per SM); + 1 producer + 1 tail warp
+constexpr int kPairConsumerWarps = 8;  // two CTAs per SM
 constexpr int kExtraWarps = 2;
 constexpr int kMailFixed = 128;       // bytes of a mailbox before its key, value and count arrays
 
@@ -68,7 +69,7 @@ __host__ __device__ inline DecodeSmem decode_smem_layout(int stages, int G, int 
 
 // dtype: 0 fp32, 1 fp16, 2 bf16.  Returns a cudaError_t as int; -1: no kernel for the shape.
 int launch_decode_fused(int dtype, int D, int G, const DecodeParams &p, int grid,
-                        int consumer_warps, cudaStream_t stream);
+                        int consumer_warps, bool wide, cudaStream_t stream);
 // Sets the dynamic shared-memory limit of the matching kernel; returns a cudaError_t as int
 // (-1: no kernel) and the CTAs per SM the occupancy calculator allows.
 int prepare_decode_fused(int dtype, int D, int G, int smem_bytes, int threads,

@@ -236,8 +236,9 @@ def test_caches_of_one_shape_and_different_budgets_coexist(zb):
     """Two live caches that use the same kernel but need different amounts of shared memory:
     creating the second must not lower the launch limit the first one needs."""
     w = wl.Workload("coexist", 1, 1, 2, 2, 128, "f16", 0, 0, 0, None, 18)
-    small = GpuCache(zb, w, np.full((1, 2), 8), np.full((1, 2), 8), np.full((1, 2), 1))
-    big = GpuCache(zb, w, np.full((1, 2), 100), np.full((1, 2), 15000), np.full((1, 2), 4))
+    small = GpuCache(zb, w, np.full((1, 2), 8), np.full((1, 2), 8), np.full((1, 2), 1), tune_ctas_per_sm=2)
+    big = GpuCache(zb, w, np.full((1, 2), 100), np.full((1, 2), 15000), np.full((1, 2), 4),
+                   tune_ctas_per_sm=2)
     try:
         # the large weight array leaves room for fewer ring stages: the cache created last asks
         # for less shared memory than the one created first
@@ -248,3 +249,14 @@ def test_caches_of_one_shape_and_different_budgets_coexist(zb):
         assert big.status() == 0 and small.status() == 0
     finally:
         big.close(), small.close()
+
+
+@pytest.mark.parametrize("ctas,warps", [(1, 16), (1, 5), (2, 8), (2, 3), (3, 4)])
+def test_launch_forms_agree(zb, oracle, ctas, warps):
+    """The wide form (one CTA per SM, up to sixteen consumer warps whose groups take tiles in
+    turn) and the paired form, with warp counts that do and do not tile a stage evenly."""
+    w = wl.Workload("forms", 1, 2, 8, 2, 128, "f16", 0, 0, 0, None, 20)
+    stats = run_decode(zb, oracle, w, np.array([[30, 60]]), np.array([[150, 41]]), np.array([[3, 5]]),
+                       steps=260, check_state_every=130, tune_ctas_per_sm=ctas,
+                       tune_consumer_warps=warps)
+    assert stats.selections > 300
