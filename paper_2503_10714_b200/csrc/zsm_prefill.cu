@@ -893,6 +893,241 @@ size_t merge_warp_smem_bytes() {
 }
 
 // ---------------------------------------------------------------------------
+// P4, blocked form (16-bit storage, B_r <= 32): the chain is still walked token by token, but
+// what a token needs from the merged keys is no longer a D-long dot product per slot.  For a
+// block of 64 evicted tokens the dot products with the merged keys as they stood at the start
+// of the block (D0 = K_blk Kr^T) and the tokens' own Gram matrix (Gm = K_blk K_blk^T) are
+// formed at once on the tensor cores.  Because a merged key is the mean of its constituents,
+//     k_r . k_t  =  ( w0_r * D0[t][r] + sum over block tokens u already merged into r of Gm[t][u] ) / w_r
+// so one warp walks the block keeping that numerator per (token, slot): per token one shared
+// load per lane, a multiply by 1/w_r, an integer warp reduction for the argmax (lowest slot wins
+// ties), and the Gram row of the token added to the chosen slot's numerators of the later
+// tokens.  After the block, every slot's key and value are rebuilt from its old mean and the
+// sum of the tokens it took.  The arithmetic is that of Eq. (hatr)/(kvr) reassociated.
+// The merged keys enter the tensor cores as three 16-bit pieces (hi + mid + lo = the fp32
+// value to its last bit), so D0 is an fp32-accumulated product of exact operands.
+// ---------------------------------------------------------------------------
+constexpr int kBlkTokens = 64;
+constexpr int kBlkNS = 33;              // row stride of the numerator table (bank-conflict free)
+constexpr int kBlkGS = kBlkTokens + 4;  // row stride of the Gram matrix
+
+template <int D>
+struct BlkSmem {
+    static constexpr int ROWB = D * 2;
+    static constexpr size_t tokK = 0;                                        // [2][64][ROWB]
+    static constexpr size_t tokV = tokK + 2 * kBlkTokens * ROWB;             // [2][64][ROWB]
+    static constexpr size_t krm = tokV + 2 * kBlkTokens * ROWB;              // [32][D] fp32
+    static constexpr size_t vrm = krm + 32 * D * 4;                          // [32][D] fp32
+    static constexpr size_t krs = vrm + 32 * D * 4;                          // [3][32][D] 16-bit
+    static constexpr size_t num = krs + 3 * 32 * ROWB;                       // [64][33] fp32
+    static constexpr size_t gm = num + kBlkTokens * kBlkNS * 4;              // [64][68] fp32
+    static constexpr size_t tgt = gm + kBlkTokens * kBlkGS * 4;              // [64] int
+    static constexpr size_t wc = tgt + kBlkTokens * 4;                       // [32] fp32 counts
+    static constexpr size_t total = wc + 32 * 4;
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const PrefillParams p) {
+    using E = Elem<T>;
+    using SM = BlkSmem<D>;
+    static_assert(sizeof(T) == 2, "16-bit storage");
+    constexpr int ROWB = D * 2;
+    constexpr int CPR = ROWB / 16;
+    constexpr int SEG = ROWB / 64;
+    constexpr int EPT = D / 32;
+    constexpr int NB = kBlkTokens;
+    extern __shared__ __align__(16) uint8_t smraw[];
+
+    const int ul = blockIdx.x;
+    const UnitDesc d = p.desc[ul];
+    const int Br = d.Br;
+    const int T_len = p.T;
+    const int n_ev = reinterpret_cast<const int32_t *>(p.ws + p.wl.counts)[ul * 4];
+    const int32_t *evl = reinterpret_cast<const int32_t *>(p.ws + p.wl.evict_list) + (size_t)ul * T_len;
+    int32_t *targets = p.dbg_targets ? p.dbg_targets + (size_t)ul * T_len : nullptr;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_warps = blockDim.x >> 5;
+    const int gq = lane >> 2, tig = lane & 3;
+
+    if (Br == 0) {
+        if (targets)
+            for (int i = tid; i < n_ev; i += blockDim.x) targets[i] = -1;  // dropped (Sec. 3.2)
+        return;
+    }
+    uint8_t *tokK = smraw + SM::tokK, *tokV = smraw + SM::tokV;
+    float *KrM = reinterpret_cast<float *>(smraw + SM::krm);
+    float *VrM = reinterpret_cast<float *>(smraw + SM::vrm);
+    uint8_t *KrS = smraw + SM::krs;
+    float *Num = reinterpret_cast<float *>(smraw + SM::num);
+    float *Gm = reinterpret_cast<float *>(smraw + SM::gm);
+    int32_t *tgt = reinterpret_cast<int32_t *>(smraw + SM::tgt);
+    float *wc = reinterpret_cast<float *>(smraw + SM::wc);
+
+    const uint8_t *Kg = static_cast<const uint8_t *>(p.K) + (size_t)ul * T_len * ROWB;
+    const uint8_t *Vg = static_cast<const uint8_t *>(p.V) + (size_t)ul * T_len * ROWB;
+
+    // element e of merged key row r as three 16-bit pieces for the tensor cores
+    auto write_split = [&](int r, int e, float x) {
+        T *s0 = reinterpret_cast<T *>(KrS) + (size_t)r * D + e;
+        const T h = E::from_float(x);
+        const float r1 = x - E::to_float(h);
+        const T m = E::from_float(r1);
+        const T l = E::from_float(r1 - E::to_float(m));
+        s0[0] = h;
+        s0[32 * D] = m;
+        s0[2 * 32 * D] = l;
+    };
+
+    // ---- fill: the first B_r evicted tokens take the free slots as they are (Alg. 1) ----
+    const int n_fill = min(Br, n_ev);
+    for (int k = tid; k < 32 * D; k += blockDim.x) {
+        const int r = k / D, e = k % D;
+        float kv = 0.f, vv = 0.f;
+        if (r < n_fill) {
+            const int t = evl[r];
+            kv = E::to_float(reinterpret_cast<const T *>(Kg + (size_t)t * ROWB)[e]);
+            vv = E::to_float(reinterpret_cast<const T *>(Vg + (size_t)t * ROWB)[e]);
+        }
+        KrM[k] = kv;
+        VrM[k] = vv;
+        write_split(r, e, kv);
+    }
+    if (tid < 32) wc[tid] = tid < n_fill ? 1.f : 0.f;
+    if (targets)
+        for (int i = tid; i < n_fill; i += blockDim.x) targets[i] = -2;
+
+    // evicted tokens i0 .. i0+nb-1 of a block into token buffer `buf`
+    auto fetch_block = [&](int i0, int buf) {
+        const int nb = min(NB, n_ev - i0);
+        for (int c = tid; c < nb * 2 * CPR; c += blockDim.x) {
+            const int tok = c / (2 * CPR), rem = c % (2 * CPR);
+            const int which = rem / CPR, cc = rem % CPR;
+            const int t = evl[i0 + tok];
+            uint8_t *dst = (which ? tokV : tokK) + ((size_t)buf * NB + tok) * ROWB + cc * 16;
+            cp_async16(dst, (which ? Vg : Kg) + (size_t)t * ROWB + cc * 16);
+        }
+        cp_async_commit();
+    };
+
+    if (n_fill < n_ev) fetch_block(n_fill, 0);
+    int buf = 0;
+    for (int i0 = n_fill; i0 < n_ev; i0 += NB, buf ^= 1) {
+        const int nb = min(NB, n_ev - i0);
+        cp_async_wait<0>();
+        __syncthreads();  // this block's tokens have landed; the previous block's update is done
+        // next block into the other buffer, whose last readers (the previous block's update) are
+        // behind the barrier above; it lands while this block is processed
+        if (i0 + NB < n_ev) fetch_block(i0 + NB, buf ^ 1);
+        const uint8_t *bK = tokK + (size_t)buf * NB * ROWB;
+        const uint8_t *bV = tokV + (size_t)buf * NB * ROWB;
+
+        // ---- bulk: D0 (16 tiles of 16 tokens x 8 slots) and Gm (32 tiles of 16 x 8 tokens) ----
+        for (int item = warp; item < 48; item += n_warps) {
+            const bool is_g = item >= 16;
+            const int it = is_g ? item - 16 : item;
+            const int mt = is_g ? it / 8 : it / 4, nt = is_g ? it % 8 : it % 4;
+            if (!is_g && nt * 8 >= Br) continue;
+            const uint8_t *pa = bK + (mt * 16 + gq) * ROWB + tig * 16;
+            float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+            const int n_split = is_g ? 1 : 3;
+            for (int sp = 0; sp < n_split; ++sp) {
+                const uint8_t *pb = (is_g ? bK : KrS + (size_t)sp * 32 * ROWB) + (nt * 8 + gq) * ROWB + tig * 16;
+#pragma unroll
+                for (int j = 0; j < SEG; ++j) {
+                    const uint4 ra = *reinterpret_cast<const uint4 *>(pa + j * 64);
+                    const uint4 rc = *reinterpret_cast<const uint4 *>(pa + 8 * ROWB + j * 64);
+                    const uint4 qb = *reinterpret_cast<const uint4 *>(pb + j * 64);
+                    mma_16x8x16<T>(c0, ra.x, rc.x, ra.y, rc.y, qb.x, qb.y);
+                    mma_16x8x16<T>(c1, ra.z, rc.z, ra.w, rc.w, qb.z, qb.w);
+                }
+            }
+            const int row = mt * 16 + gq, col = nt * 8 + tig * 2;
+            if (is_g) {
+                Gm[row * kBlkGS + col] = c0[0] + c1[0];
+                Gm[row * kBlkGS + col + 1] = c0[1] + c1[1];
+                Gm[(row + 8) * kBlkGS + col] = c0[2] + c1[2];
+                Gm[(row + 8) * kBlkGS + col + 1] = c0[3] + c1[3];
+            } else {
+                const float w0a = wc[col], w0b = wc[col + 1];
+                Num[row * kBlkNS + col] = w0a * (c0[0] + c1[0]);
+                Num[row * kBlkNS + col + 1] = w0b * (c0[1] + c1[1]);
+                Num[(row + 8) * kBlkNS + col] = w0a * (c0[2] + c1[2]);
+                Num[(row + 8) * kBlkNS + col + 1] = w0b * (c0[3] + c1[3]);
+            }
+        }
+        __syncthreads();
+
+        // ---- the chain itself, one warp: lane r watches slot r ----
+        if (warp == 0) {
+            float w = lane < Br ? wc[lane] : 1.f;
+            float rw = __frcp_rn(w);
+            for (int t = 0; t < nb; ++t) {
+                const float val = Num[t * kBlkNS + lane] * rw;  // k_r . k_t  (Eq. (hatr))
+                const uint32_t key = lane < Br ? order_key(val) : 0u;
+                const uint32_t best = __reduce_max_sync(0xffffffffu, key);
+                const int rhat = __ffs(__ballot_sync(0xffffffffu, key == best && lane < Br)) - 1;
+                if (lane == 0) tgt[t] = rhat;
+                if (lane == rhat) {
+                    w += 1.f;
+                    rw = __frcp_rn(w);
+                }
+                for (int u = t + 1 + lane; u < nb; u += 32)
+                    Num[u * kBlkNS + rhat] += Gm[t * kBlkGS + u];  // Gm is symmetric: row t
+                __syncwarp();
+            }
+        }
+        __syncthreads();
+
+        // ---- Eq. (kvr) for the whole block: slot r's mean over its old content and its takes ----
+        for (int r = warp; r < Br; r += n_warps) {
+            float sk[EPT], sv[EPT];
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) sk[e] = sv[e] = 0.f;
+            int n = 0;
+            for (int t = 0; t < nb; ++t) {
+                if (tgt[t] != r) continue;  // uniform across the warp
+                const T *kt = reinterpret_cast<const T *>(bK + (size_t)t * ROWB) + lane * EPT;
+                const T *vt = reinterpret_cast<const T *>(bV + (size_t)t * ROWB) + lane * EPT;
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) {
+                    sk[e] += E::to_float(kt[e]);
+                    sv[e] += E::to_float(vt[e]);
+                }
+                ++n;
+            }
+            if (n > 0) {
+                const float w0 = wc[r];
+                const float inv = __frcp_rn(w0 + static_cast<float>(n));
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) {
+                    const int k = r * D + lane * EPT + e;
+                    const float nk = fmaf(w0, KrM[k], sk[e]) * inv;
+                    KrM[k] = nk;
+                    VrM[k] = fmaf(w0, VrM[k], sv[e]) * inv;
+                    write_split(r, lane * EPT + e, nk);
+                }
+                __syncwarp();
+                if (lane == 0) wc[r] = w0 + static_cast<float>(n);
+            }
+        }
+        if (targets)
+            for (int t = tid; t < nb; t += blockDim.x) targets[i0 + t] = tgt[t];
+        // the next iteration's barrier orders these writes before their readers
+    }
+    __syncthreads();
+
+    const int n_res = n_fill;
+    float *Kr_g = reinterpret_cast<float *>(p.base + d.kr_off);
+    float *Vr_g = reinterpret_cast<float *>(p.base + d.vr_off);
+    uint32_t *w_g = reinterpret_cast<uint32_t *>(p.base + d.w_off);
+    for (int k = tid; k < n_res * D; k += blockDim.x) {
+        Kr_g[k] = KrM[k];
+        Vr_g[k] = VrM[k];
+    }
+    if (tid < n_res) w_g[tid] = static_cast<uint32_t>(wc[tid]);
+}
+
+// ---------------------------------------------------------------------------
 // P5: survivors into the unit's slots, ascending position; one warp per row.
 // ---------------------------------------------------------------------------
 template <typename T, int D>
@@ -957,9 +1192,12 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
     prefill_select_kernel<<<p.units, 1024, 0, stream>>>(p, scores);
     // the residual chain: merged rows in registers, one per warp, up to 128 merged slots (one
     // warp per unit when the layer has many units); the shared-memory form beyond
-    if (max_br <= 32 && p.units > 2 * p.n_sm)  // more chains than row-per-warp CTAs fit at once
+    if (max_br <= 32 && p.units > 2 * p.n_sm)  // more chains than the CTA forms fit at once
         prefill_merge_warp_kernel<T, D><<<p.units, 32, merge_warp_smem_bytes<T, D>(), stream>>>(p);
-    else if (max_br <= 32)
+    else if (max_br <= 32 && sizeof(T) == 2) {
+        if constexpr (sizeof(T) == 2)
+            prefill_merge_blocked_kernel<T, D><<<p.units, 1024, BlkSmem<D>::total, stream>>>(p);
+    } else if (max_br <= 32)
         prefill_merge_rows_kernel<T, D, 1><<<p.units, kRowMergeThreads, merge_rows_smem_bytes<T, D>(), stream>>>(p);
     else if (max_br <= 64)
         prefill_merge_rows_kernel<T, D, 2><<<p.units, kRowMergeThreads, merge_rows_smem_bytes<T, D>(), stream>>>(p);
@@ -990,6 +1228,11 @@ int prepare_all() {
                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)merge_smem_bytes<D>(prefill_max_residual(D), D * (int)sizeof(T)));
     if (e != cudaSuccess) return static_cast<int>(e);
+    if constexpr (sizeof(T) == 2) {
+        e = cudaFuncSetAttribute(prefill_merge_blocked_kernel<T, D>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BlkSmem<D>::total);
+        if (e != cudaSuccess) return static_cast<int>(e);
+    }
     e = cudaFuncSetAttribute(prefill_merge_warp_kernel<T, D>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_warp_smem_bytes<T, D>());
     return static_cast<int>(e);
