@@ -1058,22 +1058,40 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
         __syncthreads();
 
         // ---- the chain itself, one warp: lane r watches slot r ----
+        // The numerators of the current token and the next three live in registers and take
+        // their corrections there; shared memory is corrected only from four tokens ahead, so
+        // no shared-memory round trip sits between one token's argmax and the next.
         if (warp == 0) {
             float w = lane < Br ? wc[lane] : 1.f;
-            float rw = __frcp_rn(w);
+            float rw = __frcp_rn(w), rw_next = __frcp_rn(w + 1.f);
+            float n0 = Num[lane];
+            float n1 = 1 < nb ? Num[1 * kBlkNS + lane] : 0.f;
+            float n2 = 2 < nb ? Num[2 * kBlkNS + lane] : 0.f;
             for (int t = 0; t < nb; ++t) {
-                const float val = Num[t * kBlkNS + lane] * rw;  // k_r . k_t  (Eq. (hatr))
+                // independent of this token's outcome: its Gram entries with the next three
+                // tokens, and the numerator of the token three ahead
+                const float g1 = t + 1 < nb ? Gm[t * kBlkGS + t + 1] : 0.f;
+                const float g2 = t + 2 < nb ? Gm[t * kBlkGS + t + 2] : 0.f;
+                const float g3 = t + 3 < nb ? Gm[t * kBlkGS + t + 3] : 0.f;
+                float n3 = t + 3 < nb ? Num[(t + 3) * kBlkNS + lane] : 0.f;
+                const float val = n0 * rw;  // k_r . k_t  (Eq. (hatr))
                 const uint32_t key = lane < Br ? order_key(val) : 0u;
                 const uint32_t best = __reduce_max_sync(0xffffffffu, key);
                 const int rhat = __ffs(__ballot_sync(0xffffffffu, key == best && lane < Br)) - 1;
+                const bool me = lane == rhat;
                 if (lane == 0) tgt[t] = rhat;
-                if (lane == rhat) {
-                    w += 1.f;
-                    rw = __frcp_rn(w);
-                }
-                for (int u = t + 1 + lane; u < nb; u += 32)
+                w += me ? 1.f : 0.f;
+                rw = me ? rw_next : rw;
+                rw_next = __frcp_rn(w + 1.f);
+                n1 += me ? g1 : 0.f;
+                n2 += me ? g2 : 0.f;
+                n3 += me ? g3 : 0.f;
+                for (int u = t + 4 + lane; u < nb; u += 32)
                     Num[u * kBlkNS + rhat] += Gm[t * kBlkGS + u];  // Gm is symmetric: row t
                 __syncwarp();
+                n0 = n1;
+                n1 = n2;
+                n2 = n3;
             }
         }
         __syncthreads();
@@ -1084,16 +1102,23 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
 #pragma unroll
             for (int e = 0; e < EPT; ++e) sk[e] = sv[e] = 0.f;
             int n = 0;
-            for (int t = 0; t < nb; ++t) {
-                if (tgt[t] != r) continue;  // uniform across the warp
-                const T *kt = reinterpret_cast<const T *>(bK + (size_t)t * ROWB) + lane * EPT;
-                const T *vt = reinterpret_cast<const T *>(bV + (size_t)t * ROWB) + lane * EPT;
+            // which of the block's tokens went to slot r: one vote per half of the block
 #pragma unroll
-                for (int e = 0; e < EPT; ++e) {
-                    sk[e] += E::to_float(kt[e]);
-                    sv[e] += E::to_float(vt[e]);
+            for (int half = 0; half < 2; ++half) {
+                const int tt = half * 32 + lane;
+                unsigned mask = __ballot_sync(0xffffffffu, tt < nb && tgt[tt] == r);
+                while (mask) {
+                    const int t = half * 32 + __ffs(mask) - 1;
+                    mask &= mask - 1;
+                    const T *kt = reinterpret_cast<const T *>(bK + (size_t)t * ROWB) + lane * EPT;
+                    const T *vt = reinterpret_cast<const T *>(bV + (size_t)t * ROWB) + lane * EPT;
+#pragma unroll
+                    for (int e = 0; e < EPT; ++e) {
+                        sk[e] += E::to_float(kt[e]);
+                        sv[e] += E::to_float(vt[e]);
+                    }
+                    ++n;
                 }
-                ++n;
             }
             if (n > 0) {
                 const float w0 = wc[r];
