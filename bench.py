@@ -320,6 +320,8 @@ def main():
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--consumer-warps", type=int, default=0)
+    ap.add_argument("--split", type=int, default=0, choices=[0, 1, 2, 4, 8],
+                    help="CTAs per unit in launches with few units (0: library default, 1: never)")
     args = ap.parse_args()
     world, rank, local = dist_setup(args.gpus)
     w0 = wl.WORKLOADS[args.workload]
@@ -342,7 +344,7 @@ def main():
     stream = torch.cuda.current_stream()
     cfg = zb.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, bp,
                          bc, br, tune_stages=args.stages, tune_ctas_per_sm=args.ctas_per_sm,
-                         tune_consumer_warps=args.consumer_warps)
+                         tune_consumer_warps=args.consumer_warps, tune_split=args.split)
     buf = torch.empty(zb.zsm_cache_bytes(cfg), dtype=torch.uint8, device=dev)
     cache = zb.zsm_cache_create(cfg, buf)
 

@@ -87,6 +87,11 @@ typedef struct {
     int32_t tune_consumer_warps; /* compute warps per CTA: at most 8 with two CTAs per SM, 16 with
                                   * one (two more warps feed them
                                   * and write the cache update back) */
+    int32_t tune_split;          /* CTAs that share one unit in a launch with few units (each takes
+                                  * a slice of the unit's slots; a thread-block cluster): 0 = the
+                                  * library's choice (the largest of 8, 4, 2 that keeps the launch
+                                  * within the SM count, when units are at most half the SMs),
+                                  * 1 = never split, 2, 4 or 8 = at most that many */
 } zsm_config_t;
 
 /* Budget split of App. C.2: B_p = floor(tail_ratio*B); B_r = round(dense_ratio*

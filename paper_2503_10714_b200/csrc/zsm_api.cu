@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "zsm_decode.cuh"
+#include "zsm_decode_split.cuh"
 #include "zsm_prefill.cuh"
 
 using namespace zsm;
@@ -52,6 +53,9 @@ struct zsm_cache {
     struct Plan {
         int ctas_per_sm, consumer_warps, stages, smem_bytes, grid;
         bool wide;
+        // Split form, for a launch with at most half as many units as SMs: `split` CTAs (a
+        // cluster) share each unit; 0 = not used.
+        int split, split_warps, split_stages, split_smem, split_l_stride, split_kr_rows;
     } plan_all, plan_layer;
     int l_stride, br_max, br_max_pad, cap_max;
     int smem_bytes;
@@ -71,6 +75,9 @@ bool check_config(const zsm_config_t *c) {
     if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return false;
     if (!(c->softmax_scale >= 0.f)) return false;
     if (c->tune_stages < 0 || c->tune_ctas_per_sm < 0 || c->tune_consumer_warps < 0) return false;
+    if (c->tune_split != 0 && c->tune_split != 1 && c->tune_split != 2 && c->tune_split != 4 &&
+        c->tune_split != 8)
+        return false;
     const long n = (long)c->n_layers * c->n_kv_heads;
     for (long i = 0; i < n; ++i) {
         if (c->budget_p[i] < 0 || c->budget_c[i] < 0 || c->budget_r[i] < 0) return false;
@@ -361,6 +368,40 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
             pl.ctas_per_sm = std::min(pl.ctas_per_sm, occ);
         }
         pl.grid = std::min(default_grid(units, c->n_sm, pl.ctas_per_sm), 1024);
+
+        // Split form: only when nothing asks for the paired form and the launch is small.
+        pl.split = 0;
+        if (cfg->tune_split != 1 && cfg->tune_ctas_per_sm == 0 && units * 2 <= c->n_sm) {
+            const int limit = cfg->tune_split > 1 ? cfg->tune_split : kSplitMaxCluster;
+            const int warps = cfg->tune_consumer_warps > 0
+                                  ? std::min((int)cfg->tune_consumer_warps, kMaxConsumerWarps)
+                                  : kMaxConsumerWarps;
+            for (int C = kSplitMaxCluster; C >= 2 && pl.split == 0; C >>= 1) {
+                if (C > limit || units * C > c->n_sm) continue;
+                const int ls = split_l_stride(c->cap_max, c->br_max, s.esz, C);
+                // merged keys stay in shared memory on rank 0 when they are few (Eq. (hatr))
+                int kr_rows = c->br_max * s.D * 4 <= 32768 ? c->br_max : 0;
+                auto total = [&](int st) {
+                    return (int)split_smem_layout(st, s.G, s.D, s.row_bytes, ls, c->br_max_pad,
+                                                  kr_rows, warps).total;
+                };
+                int st = (kMaxSmemPerCta - total(0) - 64) / (kTileBytes + 16);
+                if (cfg->tune_stages > 0) st = std::min(st, (int)cfg->tune_stages);
+                st = std::min(st, 12);
+                while (st >= 2 && total(st) > kMaxSmemPerCta) --st;
+                if (st < 2) continue;
+                int fit = 0;
+                const int rc = prepare_decode_split(s.dtype, s.D, s.G, C, total(st),
+                                                    (warps + kExtraWarps) * 32, &fit);
+                if (rc != 0 || fit < 1) continue;
+                pl.split = C;
+                pl.split_warps = warps;
+                pl.split_stages = st;
+                pl.split_smem = total(st);
+                pl.split_l_stride = ls;
+                pl.split_kr_rows = kr_rows;
+            }
+        }
         return ZSM_OK;
     };
     {
@@ -437,6 +478,12 @@ zsm_status_t zsm_decode_launch_info(const zsm_cache_t *c, int32_t layer, int32_t
                                     int32_t *block, int32_t *dynamic_smem_bytes) {
     if (!c || layer < -1 || layer >= c->s.L) return ZSM_ERR_INVALID_ARG;
     const zsm_cache::Plan &pl = layer < 0 ? c->plan_all : c->plan_layer;
+    if (pl.split >= 2) {
+        if (grid) *grid = (layer < 0 ? c->s.n_units : c->s.upl) * pl.split;
+        if (block) *block = (pl.split_warps + kExtraWarps) * 32;
+        if (dynamic_smem_bytes) *dynamic_smem_bytes = pl.split_smem;
+        return ZSM_OK;
+    }
     if (grid) *grid = pl.grid;
     if (block) *block = (pl.consumer_warps + kExtraWarps) * 32;
     if (dynamic_smem_bytes) *dynamic_smem_bytes = pl.smem_bytes;
@@ -477,6 +524,21 @@ zsm_status_t zsm_decode_step(zsm_cache_t *c, int32_t layer, const void *q, const
     p.lambda = c->lambda;
     p.alpha = c->alpha;
     p.scale = c->scale;
+    if (pl.split >= 2) {
+        SplitParams sp;
+        sp.d = p;
+        sp.d.sched_off = nullptr;
+        sp.d.sched_desc = reinterpret_cast<const UnitDesc *>(c->base + lay.layer_desc) +
+                          (layer < 0 ? 0 : (size_t)layer * c->s.upl);
+        sp.d.stages = pl.split_stages;
+        sp.d.l_stride = pl.split_l_stride;
+        sp.n_units = layer < 0 ? c->s.n_units : c->s.upl;
+        sp.kr_rows = pl.split_kr_rows;
+        const int rs = launch_decode_split(c->s.dtype, c->s.D, c->s.G, sp, pl.split, pl.split_warps,
+                                           static_cast<cudaStream_t>(stream));
+        if (rs == -1) return ZSM_ERR_UNSUPPORTED;
+        return rs == 0 ? ZSM_OK : ZSM_ERR_CUDA;
+    }
     const int rc = launch_decode_fused(c->s.dtype, c->s.D, c->s.G, p, pl.grid, pl.consumer_warps,
                                        pl.wide, static_cast<cudaStream_t>(stream));
     if (rc == -1) return ZSM_ERR_UNSUPPORTED;

@@ -55,23 +55,28 @@ SMALL = wl.Workload("small", 2, 2, 2, 2, 64, "f32", 0, 0, 0, None, 11)
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
 @pytest.mark.parametrize("head_dim", [64, 128])
 @pytest.mark.parametrize("group", [1, 4])
-def test_decode_from_empty_all_kernel_variants(zb, oracle, dtype, head_dim, group):
-    """Every (dtype, head_dim, group) kernel: fill, first evictions, residual fill, merges."""
+@pytest.mark.parametrize("split", [0, 1])
+def test_decode_from_empty_all_kernel_variants(zb, oracle, dtype, head_dim, group, split):
+    """Every (dtype, head_dim, group) kernel, in the split form (a cluster of CTAs per unit: the
+    library's choice for so few units) and with one CTA per unit: fill, first evictions,
+    residual fill, merges."""
     w = SMALL.replace(dtype=dtype, head_dim=head_dim, n_q_heads=2 * group)
     bp = np.array([[6, 9], [4, 20]])
     bc = np.array([[7, 30], [5, 11]])
     br = np.array([[2, 3], [1, 5]])
-    stats = run_decode(zb, oracle, w, bp, bc, br, steps=90)
+    stats = run_decode(zb, oracle, w, bp, bc, br, steps=90, tune_split=split)
     assert stats.selections > 200 and stats.merges > 150
 
 
 @pytest.mark.parametrize("budgets", [(0, 5, 3), (5, 0, 2), (4, 6, 0), (1, 1, 1), (0, 1, 0), (1, 0, 1)])
-def test_degenerate_budgets(zb, oracle, budgets):
+@pytest.mark.parametrize("split", [0, 1])
+def test_degenerate_budgets(zb, oracle, budgets, split):
     """B_p = 0 (the new token competes at once), B_c = 0 (whatever leaves proximity is evicted),
-    B_r = 0 (pure eviction) and the smallest caches."""
+    B_r = 0 (pure eviction) and the smallest caches -- in the split form most CTAs of a cluster
+    then have no slot at all."""
     w = SMALL.replace(dtype="f16", head_dim=128, n_layers=1)
     bp, bc, br = (np.full((1, 2), x) for x in budgets)
-    run_decode(zb, oracle, w, bp, bc, br, steps=40, check_state_every=5)
+    run_decode(zb, oracle, w, bp, bc, br, steps=40, check_state_every=5, tune_split=split)
 
 
 @pytest.mark.parametrize("alpha,lam", [(0.0, 0.98), (0.5, 0.5), (1.0, 0.0), (1.0, 1.0)])
@@ -81,8 +86,9 @@ def test_alpha_and_lambda_range(zb, oracle, alpha, lam):
                alpha=alpha, lam=lam)
 
 
+@pytest.mark.parametrize("split", [0, 1])
 @pytest.mark.parametrize("layer_mode", [-1, "each"])
-def test_multi_tile_ragged_units(zb, oracle, layer_mode):
+def test_multi_tile_ragged_units(zb, oracle, layer_mode, split):
     """Slot pools that span several 16 KiB tiles with a ragged last tile, ragged per-head
     budgets, residual pools larger than one tile row group; both launch shapes."""
     w = wl.Workload("ragged", 2, 2, 8, 4, 128, "f16", 0, 0, 0, None, 12)
@@ -91,7 +97,7 @@ def test_multi_tile_ragged_units(zb, oracle, layer_mode):
     bp, bc, br = split_budgets(zb, tot)
     br[0, 1], br[1, 2] = 37, 0
     stats = run_decode(zb, oracle, w, bp, bc, br, steps=300, layer_mode=layer_mode,
-                       check_state_every=100)
+                       check_state_every=100, tune_split=split)
     assert stats.selections > 1000
 
 
@@ -260,3 +266,31 @@ def test_launch_forms_agree(zb, oracle, ctas, warps):
                        steps=260, check_state_every=130, tune_ctas_per_sm=ctas,
                        tune_consumer_warps=warps)
     assert stats.selections > 300
+
+
+@pytest.mark.parametrize("cluster,warps", [(2, 16), (4, 16), (8, 16), (4, 5), (8, 3)])
+def test_split_forms_agree(zb, oracle, cluster, warps):
+    """The split form at every cluster size, with warp counts that do and do not tile a stage
+    evenly: slices that end inside a tile, a rank whose share is only the merged slots, the
+    victim on any rank."""
+    w = wl.Workload("split", 1, 2, 8, 2, 128, "f16", 0, 0, 0, None, 23)
+    cache = GpuCache(zb, w, np.array([[30, 60]]), np.array([[150, 41]]), np.array([[3, 40]]),
+                     tune_split=cluster, tune_consumer_warps=warps)
+    try:
+        grid, block, _ = zb.zsm_decode_launch_info(cache.h, -1)
+        assert grid == w.batch * w.n_kv_heads * cluster and block == (warps + 2) * 32
+    finally:
+        cache.close()
+    stats = run_decode(zb, oracle, w, np.array([[30, 60]]), np.array([[150, 41]]), np.array([[3, 40]]),
+                       steps=260, check_state_every=130, tune_split=cluster,
+                       tune_consumer_warps=warps)
+    assert stats.selections > 300 and stats.merges > 100
+
+
+def test_split_form_with_a_large_residual_pool(zb, oracle):
+    """More merged slots than rank 0 keeps in shared memory for the residual argmax (they are
+    then read from global memory), spanning several fp32 tiles."""
+    w = wl.Workload("split_res", 1, 1, 4, 2, 128, "bf16", 0, 0, 0, None, 24)
+    stats = run_decode(zb, oracle, w, np.array([[10, 12]]), np.array([[60, 90]]), np.array([[70, 100]]),
+                       steps=330, check_state_every=110)
+    assert stats.merges > 150
