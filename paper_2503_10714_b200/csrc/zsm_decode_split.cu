@@ -11,8 +11,9 @@
 // does the residual fill / merge and the insertion (D6, D7) once every rank has read its last
 // tile.  By the time the output pass starts its tiles are already in the ring (they were
 // requested while the softmax exchange ran), so small groups of warps take different tiles at
-// the same time instead of all warps sharing one.  All cross-CTA waits are on mbarriers with a time limit; the cluster
-// barrier at the end keeps a CTA's shared memory alive until its peers are done with it.
+// the same time instead of all warps sharing one.  All cross-CTA waits are on mbarriers with a
+// time limit; the cluster barrier at the end keeps a CTA's shared memory alive until its peers
+// are done with it.
 #include "zsm_decode_split.cuh"
 
 #include <type_traits>
