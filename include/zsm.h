@@ -168,6 +168,31 @@ zsm_status_t zsm_prefill_compress_static(zsm_cache_t *c, int32_t layer, const vo
                                          uint8_t *dbg_evicted, int32_t *dbg_targets,
                                          zsm_stream_t stream);
 
+/* Full-history prompt scores: the scoring window of App. B taken as the whole prompt, i.e.
+ * Eq. (score) unrolled over every prompt query,
+ *   scores[b][h][t] = (1/G) sum_g sum_{tau = t}^{T-1} lambda^(T-1-tau) * a^(tau)_{g,t},
+ * with a^(tau) the causal softmax row of query tau [Eq. (att_score)] and the mean over the G
+ * query heads of kv head h [App. C.4].  A dense T x T x d contraction on the tensor cores, two
+ * passes: the log-sum-exp of every query's row, then the decayed column sums.  The result is
+ * what zsm_prefill_compress takes as `scores` (with Qw == NULL), for any layer of the cache.
+ *   K       dev [batch][n_kv_heads][T][head_dim], Q dev [batch][n_q_heads][T][head_dim],
+ *           storage dtype of the cache, 16-byte aligned; fp16 or bf16 only
+ *           (ZSM_ERR_UNSUPPORTED for fp32 storage: use the window form with W = T there).
+ *   lse     dev fp32 [batch][n_q_heads][T] or NULL: natural-log sum-exp of each query's scaled
+ *           causal logits, as a prefill attention kernel returns it; when given, the first
+ *           pass is skipped and `workspace` may be NULL.
+ *   scores  dev fp32 [batch][n_kv_heads][T], written.
+ *   workspace  dev, 256-byte aligned, zsm_prefill_scores_full_workspace_bytes(c, T) bytes
+ *           (the row statistics); caller-owned, free to reuse once the stream has passed.
+ * Errors: ZSM_ERR_INVALID_ARG (null or misaligned pointers, T < 1), ZSM_ERR_BUFFER_TOO_SMALL,
+ * ZSM_ERR_UNSUPPORTED, ZSM_ERR_CUDA.  Asynchronous on `stream`; nothing is allocated. */
+zsm_status_t zsm_prefill_scores_full_workspace_bytes(const zsm_cache_t *c, int32_t T,
+                                                     size_t *bytes);
+zsm_status_t zsm_prefill_scores_full(zsm_cache_t *c, const void *K, const void *Q,
+                                     const float *lse, int32_t T, float *scores,
+                                     void *workspace, size_t workspace_bytes,
+                                     zsm_stream_t stream);
+
 /* One decode step [Algorithm 1 with Eq. (att_score2)], one kernel launch.
  *   layer      0..n_layers-1: that layer's units; tensors have no layer dimension.
  *              -1: every layer in one launch; tensors carry a leading

@@ -30,7 +30,8 @@ DTYPE_CODE = {"f32": ZSM_F32, "f16": ZSM_F16, "bf16": ZSM_BF16,
 # every symbol include/zsm.h declares
 SYMBOLS = ["zsm_split_budget", "zsm_cache_bytes", "zsm_cache_create", "zsm_cache_reset",
            "zsm_cache_free", "zsm_prefill_workspace_bytes", "zsm_prefill_compress",
-           "zsm_prefill_compress_static", "zsm_fullkv_workspace_bytes", "zsm_fullkv_decode",
+           "zsm_prefill_compress_static", "zsm_prefill_scores_full_workspace_bytes",
+           "zsm_prefill_scores_full", "zsm_fullkv_workspace_bytes", "zsm_fullkv_decode",
            "zsm_fullkv_status",
            "zsm_decode_step", "zsm_decode_staging_bytes", "zsm_decode_step_host",
            "zsm_unit_capacity", "zsm_cache_export_unit", "zsm_cache_import_unit",
@@ -71,6 +72,8 @@ _lib.zsm_prefill_compress.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32,
                                       _vp, _vp, _vp]
 _lib.zsm_prefill_compress_static.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp,
                                              _vp, _vp]
+_lib.zsm_prefill_scores_full_workspace_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
+_lib.zsm_prefill_scores_full.argtypes = [_vp, _vp, _vp, _vp, _i32, _vp, _vp, _sz, _vp]
 _lib.zsm_decode_step.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.zsm_fullkv_workspace_bytes.argtypes = [_i32, _i32, _i32, _i32, C.POINTER(_sz)]
 _lib.zsm_fullkv_decode.argtypes = [_i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, C.c_float, _vp,
@@ -192,6 +195,22 @@ def zsm_prefill_compress_static(cache, layer, K, V, Qw, scores, T, W, dbg_scores
                                             _dev(scores), int(T), int(W), _dev(dbg_scores),
                                             _dev(dbg_evicted), _dev(dbg_targets),
                                             _stream(stream)), "zsm_prefill_compress_static")
+
+
+def zsm_prefill_scores_full_workspace_bytes(cache, T: int) -> int:
+    n = _sz()
+    _check(_lib.zsm_prefill_scores_full_workspace_bytes(cache, int(T), C.byref(n)),
+           "zsm_prefill_scores_full_workspace_bytes")
+    return n.value
+
+
+def zsm_prefill_scores_full(cache, K, Q, T, scores, workspace=None, lse=None, stream=None):
+    """Full-history prompt scores (every prompt query scores every earlier key) into `scores`
+    fp32 [batch][n_kv_heads][T]; `lse` optionally supplies the rows' log-sum-exp."""
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.zsm_prefill_scores_full(cache, _dev(K), _dev(Q), _dev(lse), int(T), _dev(scores),
+                                        _dev(workspace), nbytes, _stream(stream)),
+           "zsm_prefill_scores_full")
 
 
 def zsm_decode_step(cache, layer, q, k_new, v_new, out, victim_pos=None, merge_slot=None,

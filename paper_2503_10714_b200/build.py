@@ -8,9 +8,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzsm.so")
-SOURCES = ["zsm_api.cu", "zsm_decode.cu", "zsm_decode_split.cu", "zsm_prefill.cu", "zsm_noalloc.cu",
-           "zsm_fullkv.cu"]
-HEADERS = ["zsm_common.cuh", "zsm_decode.cuh", "zsm_decode_split.cuh", "zsm_prefill.cuh"]
+SOURCES = ["zsm_api.cu", "zsm_decode.cu", "zsm_decode_split.cu", "zsm_prefill.cu",
+           "zsm_prefill_full.cu", "zsm_noalloc.cu", "zsm_fullkv.cu"]
+HEADERS = ["zsm_common.cuh", "zsm_decode.cuh", "zsm_decode_split.cuh", "zsm_prefill.cuh",
+           "zsm_prefill_full.cuh"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -12,6 +12,7 @@
 #include "zsm_decode.cuh"
 #include "zsm_decode_split.cuh"
 #include "zsm_prefill.cuh"
+#include "zsm_prefill_full.cuh"
 
 using namespace zsm;
 
@@ -625,6 +626,45 @@ zsm_status_t zsm_prefill_compress(zsm_cache_t *c, int32_t layer, const void *K, 
     p.scale = c->scale;
     const int rc = launch_prefill(c->s.dtype, c->s.D, p, std::max(1, c->layer_br_max[layer]),
                                   static_cast<cudaStream_t>(stream));
+    if (rc == -1) return ZSM_ERR_UNSUPPORTED;
+    return rc == 0 ? ZSM_OK : ZSM_ERR_CUDA;
+}
+
+zsm_status_t zsm_prefill_scores_full_workspace_bytes(const zsm_cache_t *c, int32_t T,
+                                                     size_t *bytes) {
+    if (!c || !bytes || T < 1) return ZSM_ERR_INVALID_ARG;
+    *bytes = align_up((size_t)c->s.B * c->s.Hq * T * sizeof(float));
+    return ZSM_OK;
+}
+
+zsm_status_t zsm_prefill_scores_full(zsm_cache_t *c, const void *K, const void *Q,
+                                     const float *lse, int32_t T, float *scores,
+                                     void *workspace, size_t workspace_bytes,
+                                     zsm_stream_t stream) {
+    if (!c || !K || !Q || !scores || T < 1) return ZSM_ERR_INVALID_ARG;
+    if (!aligned16(K) || !aligned16(Q)) return ZSM_ERR_INVALID_ARG;
+    if (c->s.dtype == ZSM_F32) return ZSM_ERR_UNSUPPORTED;
+    if (!lse) {
+        size_t need = 0;
+        zsm_prefill_scores_full_workspace_bytes(c, T, &need);
+        if (!workspace || reinterpret_cast<uintptr_t>(workspace) % kAlign != 0)
+            return ZSM_ERR_INVALID_ARG;
+        if (workspace_bytes < need) return ZSM_ERR_BUFFER_TOO_SMALL;
+    }
+    if ((long)c->s.B * c->s.Hq > 65535) return ZSM_ERR_UNSUPPORTED;
+    FullScoreParams p;
+    p.K = K;
+    p.Q = Q;
+    p.lse = lse;
+    p.lse_out = lse ? nullptr : static_cast<float *>(workspace);
+    p.scores = scores;
+    p.batch = c->s.B;
+    p.n_kv_heads = c->s.Hkv;
+    p.G = c->s.G;
+    p.T = T;
+    p.lambda = c->lambda;
+    p.scale = c->scale;
+    const int rc = launch_full_scores(c->s.dtype, c->s.D, p, static_cast<cudaStream_t>(stream));
     if (rc == -1) return ZSM_ERR_UNSUPPORTED;
     return rc == 0 ? ZSM_OK : ZSM_ERR_CUDA;
 }

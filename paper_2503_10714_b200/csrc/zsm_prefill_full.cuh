@@ -1,0 +1,25 @@
+// Launch interface of the full-history prompt scoring (every prompt query scores every earlier
+// key: the W = T case of App. B, Eq. (score) unrolled over the whole prompt).
+#pragma once
+
+#include "zsm_common.cuh"
+
+namespace zsm {
+
+constexpr int kFullBlock = 64;  // queries per row block, keys per column block
+
+struct FullScoreParams {
+    const void *K;      // [batch][n_kv_heads][T][d]
+    const void *Q;      // [batch][n_q_heads][T][d]
+    const float *lse;   // [batch][n_q_heads][T] natural log-sum-exp of each query's causal row
+    float *lse_out;     // same shape, written by the first pass (null when `lse` is supplied)
+    float *scores;      // [batch][n_kv_heads][T]
+    int32_t batch, n_kv_heads, G, T;
+    float lambda, scale;
+};
+
+// Enqueues one or both passes on `stream`: row statistics (skipped when p.lse is set), then the
+// decayed column sums.  dtype: 1 fp16, 2 bf16.  Returns a cudaError_t as int; -1: no kernel.
+int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t stream);
+
+}  // namespace zsm

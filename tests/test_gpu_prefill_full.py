@@ -1,0 +1,144 @@
+"""GPU parity of the full-history prompt scores (every prompt query scores every earlier key)
+against the oracle's prompt pass with the window taken as the whole prompt, against the
+definition written out with a library softmax, and end to end into the compression."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from harness import GpuCache, ParityStats, SCORE_RTOL, f64, oracle_unit_for, prefill_check
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def zb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2503_10714_b200 import binding
+    return binding
+
+
+def full_scores(zb, cache, K, Q, lse=None):
+    T = K.shape[2]
+    w = cache.w
+    scores = torch.full((w.batch, w.n_kv_heads, T), float("nan"), dtype=torch.float32, device="cuda")
+    ws = None
+    if lse is None:
+        ws = torch.empty(zb.zsm_prefill_scores_full_workspace_bytes(cache.h, T), dtype=torch.uint8,
+                         device="cuda")
+    zb.zsm_prefill_scores_full(cache.h, K, Q, T, scores, ws, lse)
+    torch.cuda.synchronize()
+    return scores, ws
+
+
+def oracle_scores(oracle, cache, K, V, Q, b, h):
+    G = cache.w.group
+    unit = oracle_unit_for(oracle, cache, 0, h)
+    return unit.prefill_compress(f64(K[b, h]), f64(V[b, h]), Qw=f64(Q[b, h * G:(h + 1) * G])).scores
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("head_dim,group", [(64, 1), (128, 1), (128, 4), (64, 2)])
+def test_full_scores_match_the_oracle(zb, oracle, dtype, head_dim, group):
+    """Several 64-row blocks with a ragged last one, every kernel variant."""
+    T = 333
+    w = wl.Workload("full", 1, 2, 2 * group, 2, head_dim, dtype, T, 0, T, None, 31)
+    cache = GpuCache(zb, w, [[8, 12]], [[20, 30]], [[2, 3]])
+    try:
+        K, V, Q = wl.prompt(w, 0)
+        s_gpu, _ = full_scores(zb, cache, K.cuda(), Q.cuda())
+        s_gpu = s_gpu.cpu().numpy().astype(np.float64)
+        assert np.isfinite(s_gpu).all()
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                ref = oracle_scores(oracle, cache, K, V, Q, b, h).astype(np.float64)
+                rel = np.abs(s_gpu[b, h] - ref) / np.maximum(np.abs(ref), 1e-30)
+                assert rel.max() <= SCORE_RTOL, f"unit {(b, h)}: relative error {rel.max():.3e}"
+    finally:
+        cache.close()
+
+
+@pytest.mark.parametrize("T", [1, 2, 63, 64, 65, 128, 200])
+@pytest.mark.parametrize("lam", [0.98, 1.0, 0.0])
+def test_full_scores_against_the_definition(zb, T, lam):
+    """Block edges, the shortest prompts and the ends of the decay range, against the column
+    sums of a causal softmax matrix computed with torch in fp64; also with the row statistics
+    handed in instead of computed."""
+    w = wl.Workload("fulldef", 1, 1, 4, 2, 128, "f16", T, 0, T, None, 32)
+    cache = GpuCache(zb, w, [[4, 4]], [[4, 4]], [[1, 1]], lam=lam)
+    try:
+        K, V, Q = wl.prompt(w, 0)
+        s_gpu, ws = full_scores(zb, cache, K.cuda(), Q.cuda())
+        G = w.group
+        Kd, Qd = K.double(), Q.double()
+        logits = torch.einsum("bhgqd,bhkd->bhgqk", Qd.view(1, 2, G, T, 128), Kd) / np.sqrt(128.0)
+        mask = torch.tril(torch.ones(T, T, dtype=torch.bool))
+        logits = logits.masked_fill(~mask, float("-inf"))
+        A = torch.softmax(logits, dim=-1)                       # [b, h, g, query, key]
+        decay = torch.tensor([1.0 if q == T - 1 else float(lam) ** (T - 1 - q) for q in range(T)],
+                             dtype=torch.float64)
+        ref = (A * decay.view(1, 1, 1, T, 1)).sum(dim=3).mean(dim=2)  # [b, h, key]
+        got = s_gpu.cpu().double()
+        err = (got - ref).abs() / ref.abs().clamp_min(1e-30)
+        nz = ref > 0
+        assert err[nz].max().item() <= SCORE_RTOL if nz.any() else True
+        assert (got[~nz] == 0).all()
+        # the same with the log-sum-exp of each row supplied by the caller
+        lse = torch.logsumexp(logits, dim=-1).view(1, 2 * G, T).float().cuda().contiguous()
+        s2, _ = full_scores(zb, cache, K.cuda(), Q.cuda(), lse=lse)
+        err2 = (s2.cpu().double() - ref).abs() / ref.abs().clamp_min(1e-30)
+        assert err2[nz].max().item() <= SCORE_RTOL if nz.any() else True
+    finally:
+        cache.close()
+
+
+def test_full_scores_feed_the_compression(zb, oracle):
+    """Scores from the full-history pass, handed to the compression as precomputed scores, give
+    the oracle's selection, merge chain and state for a window equal to the prompt."""
+    T = 500
+    w = wl.Workload("fullpp", 1, 1, 4, 2, 128, "bf16", T, 0, T, None, 33)
+    cache = GpuCache(zb, w, [[16, 24]], [[40, 56]], [[3, 6]])
+    stats = ParityStats()
+    try:
+        K, V, Q = wl.prompt(w, 0)
+        s_gpu, _ = full_scores(zb, cache, K.cuda(), Q.cuda())
+        dbg = cache.prefill(0, K.cuda(), V.cuda(), None, s_gpu)
+        for h in range(w.n_kv_heads):
+            prefill_check(oracle, cache, 0, 0, h, K, V, Q, dbg, stats,
+                          scores_given=s_gpu[0, h].cpu().numpy(), tag=f"unit {h}")
+        assert cache.status() == 0 and stats.merges > 500
+    finally:
+        cache.close()
+
+
+def test_full_scores_argument_errors(zb):
+    w = wl.Workload("fullerr", 1, 1, 2, 2, 64, "f32", 32, 0, 32, None, 34)
+    cache = GpuCache(zb, w, [[4, 4]], [[4, 4]], [[1, 1]])
+    try:
+        K, V, Q = (t.cuda() for t in wl.prompt(w, 0))
+        s = torch.empty(1, 2, 32, dtype=torch.float32, device="cuda")
+        ws = torch.empty(zb.zsm_prefill_scores_full_workspace_bytes(cache.h, 32), dtype=torch.uint8,
+                         device="cuda")
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_prefill_scores_full(cache.h, K, Q, 32, s, ws)
+        assert e.value.status == zb.ZSM_ERR_UNSUPPORTED  # fp32 storage
+    finally:
+        cache.close()
+    w = w.replace(dtype="f16")
+    cache = GpuCache(zb, w, [[4, 4]], [[4, 4]], [[1, 1]])
+    try:
+        K, V, Q = (t.cuda() for t in wl.prompt(w, 0))
+        s = torch.empty(1, 2, 32, dtype=torch.float32, device="cuda")
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_prefill_scores_full(cache.h, K, Q, 32, s, None)
+        assert e.value.status == zb.ZSM_ERR_INVALID_ARG  # no workspace and no row statistics
+        small = torch.empty(128, dtype=torch.uint8, device="cuda")
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_prefill_scores_full(cache.h, K, Q, 32, s, small)
+        assert e.value.status == zb.ZSM_ERR_BUFFER_TOO_SMALL
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_prefill_scores_full(cache.h, K, Q, 0, s, small)
+        assert e.value.status == zb.ZSM_ERR_INVALID_ARG
+    finally:
+        cache.close()
