@@ -92,7 +92,7 @@ static zso_tok make_tok(const double *k, const double *v, int d, float s, int32_
 /* Sec. 3.4: fold an evicted token into the residual component.
  * Free slot left -> the token takes it with fusion count 1 (Alg. 1 l.13-14).
  * Otherwise Eq. (hatr): slot with the largest raw dot product k_r . k_t
- * (compared in fp32, equal values -> lowest slot), then Eq. (kvr): incremental
+ * (or, with p.cosine, its cosine form; compared in fp32, equal values -> lowest slot), then Eq. (kvr): incremental
  * mean of keys and values, and the fusion count goes up by one.
  * Returns the slot merged into, -2 for a fill, -1 when B_r = 0. */
 static int32_t residual_absorb(zso_unit *u, const double *k, const double *v, int32_t hint_slot,
@@ -119,10 +119,18 @@ static int32_t residual_absorb(zso_unit *u, const double *k, const double *v, in
     double hint_abs = 0.0;
     for (int r = 0; r < u->nr; ++r) {
         const double *kr = u->Kr + (size_t)r * d;
-        double acc = 0.0, aabs = 0.0;
+        double acc = 0.0, aabs = 0.0, nr2 = 0.0, nt2 = 0.0;
         for (int i = 0; i < d; ++i) {
             acc += kr[i] * k[i];
             aabs += fabs(kr[i] * k[i]);
+            nr2 += kr[i] * kr[i];
+            nt2 += k[i] * k[i];
+        }
+        if (u->p.cosine) {
+            /* cosine form of Eq. (hatr); a zero vector is similar to nothing */
+            const double nn = sqrt(nr2) * sqrt(nt2);
+            acc = nn > 0.0 ? acc / nn : 0.0;
+            aabs = nn > 0.0 ? aabs / nn : 0.0;
         }
         float f = (float)acc;
         if (r == hint_slot) {

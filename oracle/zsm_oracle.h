@@ -48,6 +48,9 @@ typedef struct {
     double lambda;  /* score decay, Eq. (score) */
     double alpha;   /* compensation strength, Eq. (att_score2) */
     double scale;   /* logit scale, 1/sqrt(d) in Eq. (att_score) */
+    int32_t cosine; /* 0: Eq. (hatr) as printed, raw dot product; 1: the cosine form the
+                     * paper's source carries commented out beside it,
+                     * k_r . k_t / (|k_r| |k_t|) */
 } zso_params;
 
 /* Optional guidance for the two integer decisions of a step.  A hinted choice

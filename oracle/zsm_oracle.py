@@ -40,7 +40,7 @@ def build(force: bool = False) -> str:
 class _Params(C.Structure):
     _fields_ = [("d", C.c_int32), ("G", C.c_int32), ("Bp", C.c_int32), ("Bc", C.c_int32),
                 ("Br", C.c_int32), ("lam", C.c_double), ("alpha", C.c_double),
-                ("scale", C.c_double)]
+                ("scale", C.c_double), ("cosine", C.c_int32)]
 
 
 class _Hint(C.Structure):
@@ -132,10 +132,10 @@ class PrefillResult:
 class Unit:
     """One (layer, sequence, kv-head) compressed cache, Algorithm 1 in fp64."""
 
-    def __init__(self, d, G, Bp, Bc, Br, lam=0.98, alpha=1.0, scale=None):
+    def __init__(self, d, G, Bp, Bc, Br, lam=0.98, alpha=1.0, scale=None, cosine=False):
         self.d, self.G, self.Bp, self.Bc, self.Br = int(d), int(G), int(Bp), int(Bc), int(Br)
         p = _Params(self.d, self.G, self.Bp, self.Bc, self.Br, float(lam), float(alpha),
-                    float(scale) if scale else 1.0 / np.sqrt(float(d)))
+                    float(scale) if scale else 1.0 / np.sqrt(float(d)), 1 if cosine else 0)
         self._h = lib().zso_unit_new(C.byref(p))
         if not self._h:
             raise ValueError("invalid oracle unit parameters")

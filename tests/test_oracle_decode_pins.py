@@ -334,6 +334,45 @@ def test_merge_target_is_max_raw_dot_product(oracle):
     assert w.tolist()[0] == 2
 
 
+def test_cosine_form_prefers_the_aligned_slot(oracle):
+    """The cosine form of Eq. (hatr) (commented out beside it in the paper's source): on the
+    same stream as above the better aligned short slot wins, and every merge target of a
+    random stream is the brute-force argmax of k_r.k_t / (|k_r||k_t|) over the merged keys as
+    they stood before the step."""
+    d = 4
+    u = oracle.Unit(d, 1, Bp=1, Bc=1, Br=2, lam=0.0, cosine=True)
+    q = np.array([[0.0, 0, 0, 1.0]])
+    vv = np.zeros(d)
+    toks = [np.array([10.0, 10.0, 0, -9]), np.array([1.0, 0.0, 0, -9]),
+            np.array([1.0, 0.0, 0, -8.5]), np.array([0.0, 0.0, 0, 5.0]),
+            np.array([0.0, 0.0, 0, 5.0])]
+    reps = [u.decode_step(q, k, vv)[1] for k in toks]
+    assert (reps[4].victim_pos, reps[4].merge_slot) == (2, 1)
+    Kr, _, w = u.residual()
+    np.testing.assert_allclose(Kr[1], (toks[1] + toks[2]) / 2)
+    assert w.tolist() == [1, 2]
+
+    rng = np.random.default_rng(77)
+    n, d, G = 120, 16, 2
+    qs, ks, vs = heavy_hitter_stream(rng, n, d, G)
+    ks = ks * rng.uniform(0.2, 5.0, size=(n, 1))  # very different key lengths
+    u = oracle.Unit(d, G, Bp=5, Bc=9, Br=4, cosine=True)
+    ud = oracle.Unit(d, G, Bp=5, Bc=9, Br=4)
+    merges = differ = 0
+    for t in range(n):
+        pos, _, Kt, _ = u.tokens()
+        Kr, _, _ = u.residual()
+        _, rep = u.decode_step(qs[t], ks[t], vs[t])
+        _, repd = ud.decode_step(qs[t], ks[t], vs[t])
+        if rep.merge_slot >= 0:
+            kv = Kt[list(pos).index(rep.victim_pos)]
+            cos = (Kr @ kv) / (np.linalg.norm(Kr, axis=1) * np.linalg.norm(kv))
+            assert rep.merge_slot == int(np.argmax(cos.astype(np.float32)))
+            merges += 1
+        differ += int(rep.merge_slot != repd.merge_slot)
+    assert merges > 80 and differ > 0  # and the two forms do part ways on such keys
+
+
 def test_hint_protocol(oracle):
     """A hinted choice is taken only inside the tolerance; otherwise the oracle keeps its own
     and flags the mismatch."""
