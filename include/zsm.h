@@ -92,6 +92,12 @@ typedef struct {
                                   * library's choice (the largest of 8, 4, 2 that keeps the launch
                                   * within the SM count, when units are at most half the SMs),
                                   * 1 = never split, 2, 4 or 8 = at most that many */
+    int32_t similarity;          /* how an evicted token picks its merged slot [Eq. (hatr)]:
+                                  * 0 = raw dot product k_r.k_t, as the paper prints it;
+                                  * 1 = cosine k_r.k_t / (|k_r||k_t|), the form the paper's source
+                                  * carries commented out beside it (a zero vector is similar to
+                                  * nothing).  With 1 the prompt pass runs its general merge
+                                  * kernel, whatever B_r is. */
 } zsm_config_t;
 
 /* Budget split of App. C.2: B_p = floor(tail_ratio*B); B_r = round(dense_ratio*

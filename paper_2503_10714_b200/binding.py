@@ -45,7 +45,7 @@ class ZsmConfig(C.Structure):
                 ("budget_r", C.POINTER(C.c_int32)), ("lam", C.c_float), ("alpha", C.c_float),
                 ("softmax_scale", C.c_float), ("tune_stages", C.c_int32),
                 ("tune_ctas_per_sm", C.c_int32), ("tune_consumer_warps", C.c_int32),
-                ("tune_split", C.c_int32)]
+                ("tune_split", C.c_int32), ("similarity", C.c_int32)]
 
 
 class ZsmError(RuntimeError):
@@ -132,7 +132,7 @@ def zsm_split_budget(B: int, tail_ratio: float = 0.5, dense_ratio: float = 0.02)
 
 def make_config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, dtype, budget_p, budget_c,
                 budget_r, lam=0.98, alpha=1.0, softmax_scale=0.0, tune_stages=0,
-                tune_ctas_per_sm=0, tune_consumer_warps=0, tune_split=0):
+                tune_ctas_per_sm=0, tune_consumer_warps=0, tune_split=0, similarity=0):
     """Builds a zsm_config_t; the budget arrays are kept alive on the returned object."""
     arrs = [np.ascontiguousarray(np.asarray(a, dtype=np.int32).reshape(-1))
             for a in (budget_p, budget_c, budget_r)]
@@ -140,7 +140,7 @@ def make_config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, dtype, budget_
                     int(DTYPE_CODE[dtype]), arrs[0].ctypes.data_as(_pi32),
                     arrs[1].ctypes.data_as(_pi32), arrs[2].ctypes.data_as(_pi32), float(lam),
                     float(alpha), float(softmax_scale), int(tune_stages), int(tune_ctas_per_sm),
-                    int(tune_consumer_warps), int(tune_split))
+                    int(tune_consumer_warps), int(tune_split), int(similarity))
     cfg._keep = arrs
     return cfg
 

@@ -43,6 +43,7 @@ struct Shape {
 struct zsm_cache {
     Shape s;
     float lambda, alpha, scale;
+    int cosine;                       // slot similarity: 0 raw dot product, 1 cosine
     std::vector<int32_t> Bp, Bc, Br;  // [L*Hkv]
     uint8_t *base;
     size_t bytes;
@@ -76,6 +77,7 @@ bool check_config(const zsm_config_t *c) {
     if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return false;
     if (!(c->softmax_scale >= 0.f)) return false;
     if (c->tune_stages < 0 || c->tune_ctas_per_sm < 0 || c->tune_consumer_warps < 0) return false;
+    if (c->similarity != 0 && c->similarity != 1) return false;
     if (c->tune_split != 0 && c->tune_split != 1 && c->tune_split != 2 && c->tune_split != 4 &&
         c->tune_split != 8)
         return false;
@@ -296,6 +298,7 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
     const Shape &s = c->s;
     c->lambda = cfg->lambda;
     c->alpha = cfg->alpha;
+    c->cosine = cfg->similarity;
     c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)s.D);
     const int nh = s.L * s.Hkv;
     c->Bp.assign(cfg->budget_p, cfg->budget_p + nh);
@@ -522,6 +525,7 @@ zsm_status_t zsm_decode_step(zsm_cache_t *c, int32_t layer, const void *q, const
     p.stages = pl.stages;
     p.l_stride = c->l_stride;
     p.br_max_pad = c->br_max_pad;
+    p.cosine = c->cosine;
     p.lambda = c->lambda;
     p.alpha = c->alpha;
     p.scale = c->scale;
@@ -622,6 +626,7 @@ zsm_status_t zsm_prefill_compress(zsm_cache_t *c, int32_t layer, const void *K, 
     p.n_kv_heads = c->s.Hkv;
     p.n_sm = c->n_sm;
     p.max_cap = c->layer_cap_max[layer];
+    p.cosine = c->cosine;
     p.lambda = c->lambda;
     p.scale = c->scale;
     const int rc = launch_prefill(c->s.dtype, c->s.D, p, std::max(1, c->layer_br_max[layer]),

@@ -27,6 +27,7 @@ struct DecodeParams {
     int32_t stages;              // ring depth
     int32_t l_stride;            // floats per query head in the weight array
     int32_t br_max_pad;          // largest B_r, rounded up to 4
+    int32_t cosine;              // slot similarity of Eq. (hatr): 0 raw dot product, 1 cosine
     float lambda, alpha, scale;
 };
 

@@ -375,7 +375,16 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
                     mv[e] = vc[e];
                 }
             } else {
-                // Eq. (hatr): raw dot product with every merged key; ties to the lowest slot
+                // Eq. (hatr): raw dot product with every merged key (or its cosine form);
+                // ties to the lowest slot
+                float nt2 = 0.f;
+                if (p.cosine) {
+                    nt2 = kc[0] * kc[0];
+                    nt2 = fmaf(kc[1], kc[1], nt2);
+                    nt2 = fmaf(kc[2], kc[2], nt2);
+                    nt2 = fmaf(kc[3], kc[3], nt2);
+                    nt2 = group_sum<LPR32>(nt2);
+                }
                 float bd = -INFINITY;
                 int br = 0x7fffffff;
                 for (int r0 = 0; r0 < n_res; r0 += 4 * RPW32) {
@@ -395,6 +404,15 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
                         acc = fmaf(kr[u].z, kc[2], acc);
                         acc = fmaf(kr[u].w, kc[3], acc);
                         acc = group_sum<LPR32>(acc);
+                        if (p.cosine) {
+                            float nr2 = kr[u].x * kr[u].x;
+                            nr2 = fmaf(kr[u].y, kr[u].y, nr2);
+                            nr2 = fmaf(kr[u].z, kr[u].z, nr2);
+                            nr2 = fmaf(kr[u].w, kr[u].w, nr2);
+                            nr2 = group_sum<LPR32>(nr2);
+                            const float nn = sqrtf(nr2) * sqrtf(nt2);
+                            acc = nn > 0.f ? acc / nn : 0.f;
+                        }
                         if (r < n_res && (br == 0x7fffffff || acc > bd)) {
                             bd = acc;
                             br = r;

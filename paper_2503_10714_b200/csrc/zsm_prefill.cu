@@ -497,15 +497,32 @@ __global__ void __launch_bounds__(kMergeWarps * 32) prefill_merge_kernel(const P
             }
         } else {
             float kc[EPT];
+            float nt2 = 0.f;  // |k_t|^2, for the cosine form
 #pragma unroll
-            for (int e = 0; e < EPT; ++e) kc[e] = E::to_float(kc_row[lane * EPT + e]);
+            for (int e = 0; e < EPT; ++e) {
+                kc[e] = E::to_float(kc_row[lane * EPT + e]);
+                nt2 = fmaf(kc[e], kc[e], nt2);
+            }
+            if (p.cosine) {
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) nt2 += __shfl_xor_sync(0xffffffffu, nt2, off);
+            }
             for (int r = warp; r < Br; r += kMergeWarps) {  // Eq. (hatr)
                 const float *kr = Kr_s + (size_t)r * D + lane * EPT;
-                float acc = 0.f;
+                float acc = 0.f, nr2 = 0.f;
 #pragma unroll
-                for (int e = 0; e < EPT; ++e) acc = fmaf(kr[e], kc[e], acc);
+                for (int e = 0; e < EPT; ++e) {
+                    acc = fmaf(kr[e], kc[e], acc);
+                    nr2 = fmaf(kr[e], kr[e], nr2);
+                }
 #pragma unroll
                 for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                if (p.cosine) {
+#pragma unroll
+                    for (int off = 16; off >= 1; off >>= 1) nr2 += __shfl_xor_sync(0xffffffffu, nr2, off);
+                    const float nn = sqrtf(nr2) * sqrtf(nt2);
+                    acc = nn > 0.f ? acc / nn : 0.f;
+                }
                 if (lane == 0) dots_s[r] = acc;
             }
             __syncthreads();
@@ -1217,7 +1234,10 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
     prefill_select_kernel<<<p.units, 1024, 0, stream>>>(p, scores);
     // the residual chain: merged rows in registers, one per warp, up to 128 merged slots (one
     // warp per unit when the layer has many units); the shared-memory form beyond
-    if (max_br <= 32 && p.units > 2 * p.n_sm)  // more chains than the CTA forms fit at once
+    if (p.cosine)  // the cosine variant of Eq. (hatr) is built into the general form only
+        prefill_merge_kernel<T, D><<<p.units, kMergeWarps * 32,
+                                     merge_smem_bytes<D>(max_br, D * (int)sizeof(T)), stream>>>(p);
+    else if (max_br <= 32 && p.units > 2 * p.n_sm)  // more chains than the CTA forms fit at once
         prefill_merge_warp_kernel<T, D><<<p.units, 32, merge_warp_smem_bytes<T, D>(), stream>>>(p);
     else if (max_br <= 32 && sizeof(T) == 2) {
         if constexpr (sizeof(T) == 2)

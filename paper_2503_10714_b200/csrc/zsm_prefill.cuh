@@ -57,6 +57,7 @@ struct PrefillParams {
     int32_t units, T, W, G, n_kv_heads;
     int32_t n_sm;              // SMs of the device (picks the form of the merge kernel)
     int32_t max_cap;           // largest B_p + B_c among these units
+    int32_t cosine;            // slot similarity of Eq. (hatr): 0 raw dot product, 1 cosine
     float lambda, scale;
 };
 

@@ -26,11 +26,12 @@ from . import binding as zb
 
 
 class _Cache:
-    def __init__(self, w, bp, bc, br, alpha, lam=0.98):
+    def __init__(self, w, bp, bc, br, alpha, lam=0.98, similarity=0):
         self.w = w
         full = lambda x: np.full((w.n_layers, w.n_kv_heads), int(x), dtype=np.int32)
         self.cfg = zb.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype,
-                                  full(bp), full(bc), full(br), lam=lam, alpha=alpha)
+                                  full(bp), full(bc), full(br), lam=lam, alpha=alpha,
+                                  similarity=similarity)
         self.buf = torch.empty(zb.zsm_cache_bytes(self.cfg), dtype=torch.uint8, device="cuda")
         self.h = zb.zsm_cache_create(self.cfg, self.buf)
         self.out = torch.empty(w.n_layers, w.batch, w.n_q_heads, w.head_dim, dtype=w.torch_dtype,
@@ -49,7 +50,7 @@ class _Cache:
 
 def run(ratios=(0.5, 0.2, 0.1, 0.05), prompt_len=4096, steps=128, n_layers=2, batch=2, heads=8,
         head_dim=128, dtype="f16", window=32, seed=41, tail_ratio=0.5, dense_ratio=0.02,
-        alpha=1.0, lam=0.98):
+        alpha=1.0, lam=0.98, similarity=0):
     """Mean relative output error per ratio for merging and for eviction.  Returns a dict
     {ratio: {"merge": e, "evict": e, "reduction": 1 - merge/evict, "slots": B, "B_r": r}}."""
     w = wl.Workload("error_analysis", n_layers, batch, heads, heads, head_dim, dtype, prompt_len,
@@ -62,7 +63,8 @@ def run(ratios=(0.5, 0.2, 0.1, 0.05), prompt_len=4096, steps=128, n_layers=2, ba
         B = max(4, int(round(r * prompt_len)))
         bp, bc, br = zb.zsm_split_budget(B, tail_ratio, dense_ratio)
         bp0, bc0, _ = zb.zsm_split_budget(B, tail_ratio, 0.0)
-        cands[r] = (B, br, _Cache(w, bp, bc, br, alpha, lam), _Cache(w, bp0, bc0, 0, 1.0, lam))
+        cands[r] = (B, br, _Cache(w, bp, bc, br, alpha, lam, similarity),
+                    _Cache(w, bp0, bc0, 0, 1.0, lam))
     caches = [ref] + [c for v in cands.values() for c in v[2:]]
     need = max(zb.zsm_prefill_workspace_bytes(c.h, prompt_len, window) for c in caches)
     ws = torch.empty(need, dtype=torch.uint8, device=dev)
@@ -89,8 +91,11 @@ def run(ratios=(0.5, 0.2, 0.1, 0.05), prompt_len=4096, steps=128, n_layers=2, ba
 def sweep(ratio=0.1, **kw):
     """The paper's sensitivity axes (App. C.2) through the same kernels, on synthetic data: mean
     relative output error of the merging cache at one cache ratio while one setting varies --
-    B_p/B, B_r/(B - B_p), alpha, lambda.  Returns {axis: {value: error}}."""
-    out = {"tail_ratio": {}, "dense_ratio": {}, "alpha": {}, "lambda": {}}
+    B_p/B, B_r/(B - B_p), alpha, lambda, and the slot similarity of Eq. (hatr) (raw dot product
+    or its cosine form).  Returns {axis: {value: error}}."""
+    out = {"tail_ratio": {}, "dense_ratio": {}, "alpha": {}, "lambda": {}, "similarity": {}}
+    for name, sim in (("dot", 0), ("cosine", 1)):
+        out["similarity"][name] = run(ratios=(ratio,), similarity=sim, **kw)[ratio]["merge"]
     for t in (0.1, 0.3, 0.5, 0.7, 0.9):
         out["tail_ratio"][t] = run(ratios=(ratio,), tail_ratio=t, **kw)[ratio]["merge"]
     for dr in (0.0, 0.01, 0.02, 0.05, 0.1, 0.2):

@@ -43,6 +43,7 @@ class GpuCache:
         self.bc = np.asarray(bc, np.int32).reshape(w.n_layers, w.n_kv_heads)
         self.br = np.asarray(br, np.int32).reshape(w.n_layers, w.n_kv_heads)
         self.lam, self.alpha = lam, alpha
+        self.similarity = int(tune.get("similarity", 0))
         self.cfg = zb.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim,
                                   w.dtype, self.bp, self.bc, self.br, lam, alpha, scale, **tune)
         nbytes = zb.zsm_cache_bytes(self.cfg)
@@ -132,7 +133,7 @@ def oracle_unit_for(oracle, cache: GpuCache, layer, h):
     w = cache.w
     return oracle.Unit(w.head_dim, w.group, int(cache.bp[layer, h]), int(cache.bc[layer, h]),
                        int(cache.br[layer, h]), lam=float(np.float32(cache.lam)),
-                       alpha=float(np.float32(cache.alpha)))
+                       alpha=float(np.float32(cache.alpha)), cosine=bool(cache.similarity))
 
 
 def oracle_step_check(unit, q, k, v, out_gpu, vic_gpu, slot_gpu, dtype, stats: ParityStats, tag=""):

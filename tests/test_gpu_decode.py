@@ -294,3 +294,13 @@ def test_split_form_with_a_large_residual_pool(zb, oracle):
     stats = run_decode(zb, oracle, w, np.array([[10, 12]]), np.array([[60, 90]]), np.array([[70, 100]]),
                        steps=330, check_state_every=110)
     assert stats.merges > 150
+
+
+@pytest.mark.parametrize("split", [0, 1])
+def test_cosine_slot_similarity(zb, oracle, split):
+    """The cosine form of Eq. (hatr) in both decode kernels (heavy-hitter keys are longer than
+    ordinary ones, so the two forms do not always agree)."""
+    w = wl.Workload("cosine", 1, 2, 4, 2, 128, "f16", 0, 0, 0, None, 27)
+    stats = run_decode(zb, oracle, w, np.array([[6, 10]]), np.array([[20, 31]]), np.array([[4, 9]]),
+                       steps=220, check_state_every=110, tune_split=split, similarity=1)
+    assert stats.merges > 300

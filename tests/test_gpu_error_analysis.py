@@ -32,3 +32,16 @@ def test_compensation_term_is_what_makes_merging_pay():
     e1 = error_analysis.run(alpha=1.0, **kw)[0.1]
     e0 = error_analysis.run(alpha=0.0, **kw)[0.1]
     assert e1["merge"] < 0.6 * e0["merge"] and e0["merge"] > 0.8 * e0["evict"]
+
+
+def test_cosine_similarity_variant_runs_through_the_same_kernels():
+    """Sensitivity axis "slot similarity" (the cosine form beside Eq. (hatr)): merging still
+    beats eviction, and the figure is its own (the variant is not silently the default)."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2503_10714_b200 import error_analysis
+    kw = dict(ratios=(0.1,), prompt_len=2048, steps=48)
+    dot = error_analysis.run(similarity=0, **kw)[0.1]
+    cos = error_analysis.run(similarity=1, **kw)[0.1]
+    assert 0.0 < cos["merge"] < cos["evict"]
+    assert cos["evict"] == dot["evict"] and cos["merge"] != dot["merge"]

@@ -168,3 +168,16 @@ def test_workload_c2_full(zb, oracle):
     assert stats.steps == 32 * 256
     assert stats.victim_near_ties + stats.merge_near_ties <= 64
     print("c2", stats)
+
+
+@pytest.mark.parametrize("br", [5, 70])
+def test_prompt_pass_cosine_slot_similarity(zb, oracle, br):
+    """The cosine form of Eq. (hatr) in the prompt pass (general merge kernel whatever B_r)."""
+    w = wl.Workload("ppcos", 1, 1, 4, 2, 128, "bf16", 900, 0, 16, None, 28)
+    cache = GpuCache(zb, w, [[20, 32]], [[30, 50]], [[br, br + 3]], similarity=1)
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats)
+        assert cache.status() == 0 and stats.merges > 1000
+    finally:
+        cache.close()
