@@ -301,6 +301,45 @@ def fullkv_comparator(zb, w, dev, u, stream, budget_bytes=60e9, steps=10):
             "bytes_per_step_all_layers": int(nbytes * w.n_layers / n_l)}
 
 
+# ----------------------------------------------------------------------------- full-history scoring leg
+def full_history_scores(zb, cache, w, dev, u, stream):
+    """Prompt scores with the window taken as the whole prompt (one layer): both tensor-core
+    passes, and the column-sum pass alone with the rows' log-sum-exp supplied.  Queries are
+    synthetic (the prompt generator makes only the last `window` of them)."""
+    T = w.prompt_len
+    Kp, _, _ = wl.prompt(w, 0, dev, u)
+    g = torch.Generator(device=dev)
+    g.manual_seed(w.seed * 1000003 + 17)
+    Q = torch.randn(w.batch, w.n_q_heads, T, w.head_dim, device=dev, generator=g).to(w.torch_dtype)
+    scores = torch.empty(w.batch, w.n_kv_heads, T, dtype=torch.float32, device=dev)
+    ws = torch.empty(zb.zsm_prefill_scores_full_workspace_bytes(cache, T), dtype=torch.uint8, device=dev)
+    lse = ws.view(torch.float32)[: w.batch * w.n_q_heads * T]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    for rep in range(2):  # first round warms up
+        ev[0].record(stream)
+        zb.zsm_prefill_scores_full(cache, Kp, Q, T, scores, ws)
+        ev[1].record(stream)
+        zb.zsm_prefill_scores_full(cache, Kp, Q, T, scores, None, lse)
+        ev[2].record(stream)
+        ev[2].synchronize()
+    ms_both, ms_col = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    nb = (T + 63) // 64
+    flop = 2.0 * w.batch * w.n_q_heads * (nb * (nb + 1) / 2) * 64 * 64 * w.head_dim  # per pass, causal blocks
+    tf = measured_tensor_peak()
+    return {"what": "full-history prompt scores (W = T), one layer: row log-sum-exp + decayed column sums",
+            "T": T, "ms_both_passes": ms_both, "ms_column_pass": ms_col,
+            "tflops": 2 * flop / (ms_both * 1e-3) / 1e12, "peak_tflops": tf,
+            "frac": (2 * flop / (ms_both * 1e-3) / 1e12) / tf if tf else None, "bound": "tensor"}
+
+
+def measured_tensor_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"])
+    except Exception:
+        return 1590.0
+
+
 # ----------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -432,6 +471,10 @@ def main():
     if world == 1 and not args.no_fullkv and w.dtype != "f32":
         fullkv = fullkv_comparator(zb, w, dev, u, stream)
 
+    full_hist = None
+    if world == 1 and not args.no_fullkv and w.dtype != "f32":
+        full_hist = full_history_scores(zb, cache, w, dev, u, stream)
+
     # ---- roofline of the dominant (only) kernel of the timed region ----
     n_live = (bp + bc).astype(np.int64)      # every unit is full after a 54k prompt
     n_res = br.astype(np.int64)
@@ -472,6 +515,8 @@ def main():
     }
     if per_layer is not None:
         line["per_layer_launches"] = per_layer
+    if full_hist is not None:
+        line["prompt_scores_full_history"] = full_hist
     if fullkv is not None:
         fullkv["compressed_speedup"] = fullkv["ms_per_step"] / ms_per_step
         line["fullkv"] = fullkv

@@ -3,13 +3,14 @@
 // prompt; Eq. (score) unrolled).  A dense T x T x d contraction done twice on the tensor cores:
 //   pass 1  row statistics: log-sum-exp of every query's causal row (skipped when the caller
 //           hands in the values its own prefill attention produced);
-//   pass 2  column sums: for a block of 64 keys, over every later query block and every query
+//   pass 2  column sums: for a block of 128 keys, over every later query tile and every query
 //           head of the group, exp(logit - lse) weighted by the decay.
-// Both passes are one kernel: a 64-row block of one operand stays in registers as A fragments
+// Both passes are one kernel: a 128-row block of one operand stays in registers as A fragments
 // (queries in pass 1, keys in pass 2), 64-row tiles of the other stream through a padded,
-// double-buffered shared-memory stage (cp.async) and are read as B fragments with ldmatrix;
-// each of the four warps owns 16 resident rows and reduces along the streamed index in
-// registers, so nothing but the final per-row value leaves a thread.
+// double-buffered shared-memory stage (cp.async) and are read as B fragments with ldmatrix,
+// each fragment feeding the warp's two 16-row tiles; each of the four warps owns 32 resident
+// rows and reduces along the streamed index in registers, so nothing but the final per-row
+// value leaves a thread.
 #include "zsm_prefill_full.cuh"
 
 namespace zsm {
@@ -46,14 +47,16 @@ __global__ void __launch_bounds__(kFullThreads) full_pass_kernel(const FullScore
     constexpr int TILE = kFullBlock * STRIDE;
     constexpr int KS = D / 16;          // tensor-core steps along the head dimension
     constexpr int CPR = D * 2 / 16;     // 16-byte chunks per row
+    constexpr int MT = kFullResident / 64;  // 16-row tiles of the resident block per warp
     extern __shared__ __align__(128) uint8_t smem[];
     float *off_s = reinterpret_cast<float *>(smem + 2 * TILE);  // [2][64]: pass 2, per query
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tig = lane & 3;
     const int Tn = p.T, G = p.G;
-    const int nb = (Tn + kFullBlock - 1) / kFullBlock;
-    const int rb = blockIdx.x;  // the resident block
+    const int nb = (Tn + kFullBlock - 1) / kFullBlock;  // streamed tiles that hold a position
+    const int rb = blockIdx.x;                           // the resident block
+    constexpr int RPS = kFullResident / kFullBlock;      // streamed tiles per resident block
     int b, hk, hq = 0;
     if (COLSUM) {
         b = blockIdx.y / p.n_kv_heads;
@@ -67,29 +70,33 @@ __global__ void __launch_bounds__(kFullThreads) full_pass_kernel(const FullScore
     const T *Qb = static_cast<const T *>(p.Q) + (size_t)b * p.n_kv_heads * G * Tn * D;
     const T *res = COLSUM ? Kh : Qb + (size_t)hq * Tn * D;
 
-    // resident rows of this thread: gq and gq + 8 of the warp's 16
-    const int row0 = rb * kFullBlock + warp * 16 + gq, row1 = row0 + 8;
-    uint32_t a[KS][4];
-    {
-        const T *r0p = res + (size_t)min(row0, Tn - 1) * D, *r1p = res + (size_t)min(row1, Tn - 1) * D;
+    // resident rows of this thread: gq and gq + 8 of each of the warp's MT 16-row tiles
+    const int rbase = rb * kFullResident + warp * (16 * MT) + gq;
+    uint32_t a[MT][KS][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        const T *r0p = res + (size_t)min(rbase + 16 * mt, Tn - 1) * D;
+        const T *r1p = res + (size_t)min(rbase + 16 * mt + 8, Tn - 1) * D;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            a[ks][0] = *reinterpret_cast<const uint32_t *>(r0p + 16 * ks + 2 * tig);
-            a[ks][1] = *reinterpret_cast<const uint32_t *>(r1p + 16 * ks + 2 * tig);
-            a[ks][2] = *reinterpret_cast<const uint32_t *>(r0p + 16 * ks + 8 + 2 * tig);
-            a[ks][3] = *reinterpret_cast<const uint32_t *>(r1p + 16 * ks + 8 + 2 * tig);
+            a[mt][ks][0] = *reinterpret_cast<const uint32_t *>(r0p + 16 * ks + 2 * tig);
+            a[mt][ks][1] = *reinterpret_cast<const uint32_t *>(r1p + 16 * ks + 2 * tig);
+            a[mt][ks][2] = *reinterpret_cast<const uint32_t *>(r0p + 16 * ks + 8 + 2 * tig);
+            a[mt][ks][3] = *reinterpret_cast<const uint32_t *>(r1p + 16 * ks + 8 + 2 * tig);
         }
     }
 
-    // streamed items: pass 1 key blocks 0..rb; pass 2 query blocks rb..nb-1 for each head of the group
-    const int per = COLSUM ? nb - rb : rb + 1;
+    // streamed tiles: pass 1 key tiles 0 .. the resident block's last row; pass 2 query tiles
+    // from the resident block's first row to the end, for each head of the group
+    const int first = COLSUM ? rb * RPS : 0;
+    const int per = COLSUM ? nb - first : min(rb * RPS + RPS, nb);
     const int items = COLSUM ? per * G : per;
     const float scale2 = p.scale * kLog2e;
     const float l2lam = log2f(p.lambda);
 
     auto stage_item = [&](int i, int s) {
         const int g = COLSUM ? i / per : 0;
-        const int jb = COLSUM ? rb + i % per : i;
+        const int jb = first + (COLSUM ? i % per : i);
         const T *src = COLSUM ? Qb + (size_t)(hk * G + g) * Tn * D : Kh;
         uint8_t *dst = smem + s * TILE;
         for (int c = tid; c < kFullBlock * CPR; c += kFullThreads) {
@@ -111,8 +118,15 @@ __global__ void __launch_bounds__(kFullThreads) full_pass_kernel(const FullScore
         cp_async_commit();
     };
 
-    float m[2] = {-INFINITY, -INFINITY}, z[2] = {0.f, 0.f};  // pass 1: running max / sum (log2 domain)
-    float colsum[2] = {0.f, 0.f};                             // pass 2
+    float m[MT][2], z[MT][2], colsum[MT][2];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            m[mt][h] = -INFINITY;  // pass 1: running max / sum (log2 domain)
+            z[mt][h] = 0.f;
+            colsum[mt][h] = 0.f;   // pass 2
+        }
     stage_item(0, 0);
     for (int i = 0; i < items; ++i) {
         const int s = i & 1;
@@ -123,92 +137,112 @@ __global__ void __launch_bounds__(kFullThreads) full_pass_kernel(const FullScore
             cp_async_wait<0>();
         }
         __syncthreads();
-        const int jb = COLSUM ? rb + i % per : i;
+        const int jb = first + (COLSUM ? i % per : i);
         const uint8_t *tile = smem + s * TILE;
-        float c[8][4];
+        // tiles that overlap the resident block's own positions need the causal test
+        const bool diag = jb >= rb * RPS && jb < rb * RPS + RPS;
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+        for (int hf = 0; hf < 2; ++hf) {  // half a tile (4 column tiles of 8) at a time
+            float c[MT][4][4];
 #pragma unroll
-            for (int kq = 0; kq < D / 32; ++kq) {
-                uint32_t r[4];
-                ldmatrix_x4(r, tile + (nt * 8 + (lane & 7)) * STRIDE + (kq * 4 + (lane >> 3)) * 16);
-                mma_16x8x16<T>(c[nt], a[2 * kq][0], a[2 * kq][1], a[2 * kq][2], a[2 * kq][3], r[0], r[1]);
-                mma_16x8x16<T>(c[nt], a[2 * kq + 1][0], a[2 * kq + 1][1], a[2 * kq + 1][2], a[2 * kq + 1][3], r[2], r[3]);
-            }
-        }
-        const bool diag = jb == rb;
-        if (!COLSUM) {
-            // streamed index = key; resident rows = queries; keep key <= query
-            float bm[2] = {-INFINITY, -INFINITY};
+            for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
+                for (int n4 = 0; n4 < 4; ++n4) c[mt][n4][0] = c[mt][n4][1] = c[mt][n4][2] = c[mt][n4][3] = 0.f;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v = c[nt][e] * scale2;
-                    if (diag) {
-                        const int key = jb * kFullBlock + nt * 8 + 2 * tig + (e & 1);
-                        if (key > ((e >> 1) ? row1 : row0)) v = -INFINITY;
+            for (int n4 = 0; n4 < 4; ++n4) {
+                const int nt = hf * 4 + n4;
+#pragma unroll
+                for (int kq = 0; kq < D / 32; ++kq) {
+                    uint32_t r[4];
+                    ldmatrix_x4(r, tile + (nt * 8 + (lane & 7)) * STRIDE + (kq * 4 + (lane >> 3)) * 16);
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        mma_16x8x16<T>(c[mt][n4], a[mt][2 * kq][0], a[mt][2 * kq][1], a[mt][2 * kq][2],
+                                       a[mt][2 * kq][3], r[0], r[1]);
+                        mma_16x8x16<T>(c[mt][n4], a[mt][2 * kq + 1][0], a[mt][2 * kq + 1][1],
+                                       a[mt][2 * kq + 1][2], a[mt][2 * kq + 1][3], r[2], r[3]);
                     }
-                    c[nt][e] = v;
-                    bm[e >> 1] = fmaxf(bm[e >> 1], v);
                 }
             }
+            if (!COLSUM) {
+                // streamed index = key; resident rows = queries; keep key <= query
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const float mn = fmaxf(m[h], bm[h]);
-                const float mu = mn == -INFINITY ? 0.f : mn;
-                float sum = z[h] * ex2(m[h] - mu);
+                for (int mt = 0; mt < MT; ++mt) {
+                    float bm[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) sum += ex2(c[nt][2 * h] - mu) + ex2(c[nt][2 * h + 1] - mu);
-                z[h] = sum;
-                m[h] = mn;
-            }
-        } else {
-            // streamed index = query; resident rows = keys; keep query >= key
-            const float *off = off_s + s * kFullBlock;
+                    for (int n4 = 0; n4 < 4; ++n4) {
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                const float2 o = *reinterpret_cast<const float2 *>(off + nt * 8 + 2 * tig);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v = ex2(fmaf(c[nt][e], scale2, (e & 1) ? o.y : o.x));
-                    if (diag) {
-                        const int q = jb * kFullBlock + nt * 8 + 2 * tig + (e & 1);
-                        if (q < ((e >> 1) ? row1 : row0)) v = 0.f;
+                        for (int e = 0; e < 4; ++e) {
+                            float v = c[mt][n4][e] * scale2;
+                            if (diag) {
+                                const int key = jb * kFullBlock + (hf * 4 + n4) * 8 + 2 * tig + (e & 1);
+                                if (key > rbase + 16 * mt + 8 * (e >> 1)) v = -INFINITY;
+                            }
+                            c[mt][n4][e] = v;
+                            bm[e >> 1] = fmaxf(bm[e >> 1], v);
+                        }
                     }
-                    colsum[e >> 1] += v;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const float mn = fmaxf(m[mt][h], bm[h]);
+                        const float mu = mn == -INFINITY ? 0.f : mn;
+                        float sum = z[mt][h] * ex2(m[mt][h] - mu);
+#pragma unroll
+                        for (int n4 = 0; n4 < 4; ++n4)
+                            sum += ex2(c[mt][n4][2 * h] - mu) + ex2(c[mt][n4][2 * h + 1] - mu);
+                        z[mt][h] = sum;
+                        m[mt][h] = mn;
+                    }
+                }
+            } else {
+                // streamed index = query; resident rows = keys; keep query >= key
+                const float *off = off_s + s * kFullBlock;
+#pragma unroll
+                for (int n4 = 0; n4 < 4; ++n4) {
+                    const float2 o = *reinterpret_cast<const float2 *>(off + (hf * 4 + n4) * 8 + 2 * tig);
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float v = ex2(fmaf(c[mt][n4][e], scale2, (e & 1) ? o.y : o.x));
+                            if (diag) {
+                                const int q = jb * kFullBlock + (hf * 4 + n4) * 8 + 2 * tig + (e & 1);
+                                if (q < rbase + 16 * mt + 8 * (e >> 1)) v = 0.f;
+                            }
+                            colsum[mt][e >> 1] += v;
+                        }
+                    }
                 }
             }
         }
         __syncthreads();  // the stage is refilled two items from now
     }
 
-    if (!COLSUM) {
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
+            const int row = rbase + 16 * mt + 8 * h;
+            if (!COLSUM) {
+                float mm = m[mt][h], zz = z[mt][h];
 #pragma unroll
-            for (int x = 1; x <= 2; x <<= 1) {
-                const float mo = __shfl_xor_sync(0xffffffffu, m[h], x);
-                const float zo = __shfl_xor_sync(0xffffffffu, z[h], x);
-                const float mn = fmaxf(m[h], mo);
-                const float mu = mn == -INFINITY ? 0.f : mn;
-                z[h] = z[h] * ex2(m[h] - mu) + zo * ex2(mo - mu);
-                m[h] = mn;
+                for (int x = 1; x <= 2; x <<= 1) {
+                    const float mo = __shfl_xor_sync(0xffffffffu, mm, x);
+                    const float zo = __shfl_xor_sync(0xffffffffu, zz, x);
+                    const float mn = fmaxf(mm, mo);
+                    const float mu = mn == -INFINITY ? 0.f : mn;
+                    zz = zz * ex2(mm - mu) + zo * ex2(mo - mu);
+                    mm = mn;
+                }
+                if (tig == 0 && row < Tn)
+                    p.lse_out[((size_t)b * p.n_kv_heads * G + hq) * Tn + row] = (mm + log2f(zz)) * kLn2;
+            } else {
+                float v = colsum[mt][h];
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                if (tig == 0 && row < Tn)
+                    p.scores[((size_t)b * p.n_kv_heads + hk) * Tn + row] = v * (1.0f / static_cast<float>(G));
             }
-            const int row = h ? row1 : row0;
-            if (tig == 0 && row < Tn)
-                p.lse_out[((size_t)b * p.n_kv_heads * G + hq) * Tn + row] = (m[h] + log2f(z[h])) * kLn2;
-        }
-    } else {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float v = colsum[h];
-            v += __shfl_xor_sync(0xffffffffu, v, 1);
-            v += __shfl_xor_sync(0xffffffffu, v, 2);
-            const int row = h ? row1 : row0;
-            if (tig == 0 && row < Tn)
-                p.scores[((size_t)b * p.n_kv_heads + hk) * Tn + row] = v * (1.0f / static_cast<float>(G));
         }
     }
 }
@@ -216,16 +250,16 @@ __global__ void __launch_bounds__(kFullThreads) full_pass_kernel(const FullScore
 template <typename T, int D>
 int launch_full_one(const FullScoreParams &p, cudaStream_t stream) {
     constexpr int SMEM = 2 * kFullBlock * (D * 2 + 16) + 2 * kFullBlock * 4;
-    const int nb = (p.T + kFullBlock - 1) / kFullBlock;
+    const int nres = (p.T + kFullResident - 1) / kFullResident;
     FullScoreParams q = p;
     if (!p.lse) {
-        const dim3 grid(nb, p.batch * p.n_kv_heads * p.G);
+        const dim3 grid(nres, p.batch * p.n_kv_heads * p.G);
         full_pass_kernel<T, D, false><<<grid, kFullThreads, SMEM, stream>>>(q);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return static_cast<int>(e);
         q.lse = p.lse_out;
     }
-    const dim3 grid(nb, p.batch * p.n_kv_heads);
+    const dim3 grid(nres, p.batch * p.n_kv_heads);
     full_pass_kernel<T, D, true><<<grid, kFullThreads, SMEM, stream>>>(q);
     return static_cast<int>(cudaGetLastError());
 }

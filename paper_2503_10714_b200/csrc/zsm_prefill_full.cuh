@@ -6,7 +6,8 @@
 
 namespace zsm {
 
-constexpr int kFullBlock = 64;  // queries per row block, keys per column block
+constexpr int kFullBlock = 64;      // rows of a streamed tile
+constexpr int kFullResident = 128;  // rows of the block a CTA keeps in registers
 
 struct FullScoreParams {
     const void *K;      // [batch][n_kv_heads][T][d]
