@@ -323,8 +323,8 @@ def full_history_scores(zb, cache, w, dev, u, stream):
         ev[2].record(stream)
         ev[2].synchronize()
     ms_both, ms_col = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
-    nb = (T + 63) // 64
-    flop = 2.0 * w.batch * w.n_q_heads * (nb * (nb + 1) / 2) * 64 * 64 * w.head_dim  # per pass, causal blocks
+    nres = (T + 127) // 128  # per pass: resident block rb meets 2 rb + 2 streamed tiles of 64 rows
+    flop = 2.0 * w.batch * w.n_q_heads * (nres * (nres + 1)) * 128 * 64 * w.head_dim
     tf = measured_tensor_peak()
     return {"what": "full-history prompt scores (W = T), one layer: row log-sum-exp + decayed column sums",
             "T": T, "ms_both_passes": ms_both, "ms_column_pass": ms_col,
