@@ -27,7 +27,7 @@ def zb():
     return binding
 
 
-def run_full_size(zb, oracle, w, n_sample, steps, seed=0):
+def run_full_size(zb, oracle, w, n_sample, steps, seed=0, layer_mode=-1):
     dev = "cuda"
     totals = wl.head_budgets(w)
     bp, bc, br = split_budgets(zb, totals)
@@ -69,7 +69,7 @@ def run_full_size(zb, oracle, w, n_sample, steps, seed=0):
         vic_all_min = torch.zeros((), dtype=torch.int32, device=dev)
         for step in range(steps):
             q, k, v = wl.decode_inputs(w, step, dev, u)
-            out, vic, slot = cache.decode(q, k, v, layer=-1)
+            out, vic, slot = cache.decode(q, k, v, layer=layer_mode)
             qv = q.view(w.n_layers, w.batch, w.n_kv_heads, G, w.head_dim)
             ov = out.view(w.n_layers, w.batch, w.n_kv_heads, G, w.head_dim)
             q_rec[step], o_rec[step] = qv[li, bi, hi_], ov[li, bi, hi_]
@@ -127,7 +127,7 @@ class _Shift:
     def __init__(self, cache, b0, h0):
         self.c, self.b0, self.h0 = cache, b0, h0
         self.w = cache.w
-        self.lam, self.alpha = cache.lam, cache.alpha
+        self.lam, self.alpha, self.similarity = cache.lam, cache.alpha, cache.similarity
         self.bp = cache.bp[:, h0:h0 + 1]
         self.bc = cache.bc[:, h0:h0 + 1]
         self.br = cache.br[:, h0:h0 + 1]
@@ -159,3 +159,18 @@ def test_c5_gqa_ragged(zb, oracle):
     drawn in [64, 2048]: the smallest and the largest head are always in the sample."""
     stats = run_full_size(zb, oracle, wl.C5, n_sample=8, steps=wl.C5.decode_steps)
     assert stats.steps == 8 * 512
+
+
+@pytest.mark.parametrize("w,steps", [(wl.C4_5, 256), (wl.C5, 128)], ids=["c4_5pct", "c5"])
+def test_per_layer_launches_at_full_size(zb, oracle, w, steps):
+    """The launch shape of the benchmark's per-layer leg: one launch per layer, which at these
+    sizes is the split form (a cluster of 4 CTAs per unit for c4's 32 units per layer, of 2 for
+    c5's 64)."""
+    cache = GpuCache(zb, w.replace(n_layers=1), *split_budgets(zb, wl.head_budgets(w)[:1]))
+    try:
+        grid, _, _ = zb.zsm_decode_launch_info(cache.h, 0)
+        assert grid > w.batch * w.n_kv_heads, "expected several CTAs per unit"
+    finally:
+        cache.close()
+    stats = run_full_size(zb, oracle, w, n_sample=4, steps=steps, seed=3, layer_mode="each")
+    assert stats.steps == 4 * steps
