@@ -335,7 +335,8 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
         delete c;
         return ZSM_ERR_UNSUPPORTED;
     }
-    if (prepare_prefill(s.dtype, s.D) != 0) {
+    if (prepare_prefill(s.dtype, s.D) != 0 ||
+        (s.dtype != ZSM_F32 && prepare_full_scores(s.dtype, s.D) != 0)) {
         delete c;
         return ZSM_ERR_CUDA;
     }
@@ -663,6 +664,7 @@ zsm_status_t zsm_prefill_scores_full(zsm_cache_t *c, const void *K, const void *
     p.lse = lse;
     p.lse_out = lse ? nullptr : static_cast<float *>(workspace);
     p.scores = scores;
+    p.status = reinterpret_cast<int32_t *>(c->base + c->lay.status);
     p.batch = c->s.B;
     p.n_kv_heads = c->s.Hkv;
     p.G = c->s.G;

@@ -5,58 +5,145 @@
 //           hands in the values its own prefill attention produced);
 //   pass 2  column sums: for a block of 128 keys, over every later query tile and every query
 //           head of the group, exp(logit - lse) weighted by the decay.
-// Both passes are one kernel: a 128-row block of one operand stays in registers as A fragments
-// (queries in pass 1, keys in pass 2), 64-row tiles of the other stream through a padded,
-// double-buffered shared-memory stage (cp.async) and are read as B fragments with ldmatrix,
-// each fragment feeding the warp's two 16-row tiles; each of the four warps owns 32 resident
-// rows and reduces along the streamed index in registers, so nothing but the final per-row
-// value leaves a thread.
+// Both passes are one kernel.  A 128-row block of one operand (queries in pass 1, keys in pass 2)
+// stays in shared memory; 128-row tiles of the other stream through a three-stage ring, brought in
+// by TMA (cp.async.bulk.tensor, 128-byte swizzle) on full / free mbarriers.  One thread issues
+// tcgen05.mma: 128 x 128 x d logits per tile, both operands from shared memory, the fp32
+// accumulator in tensor memory, two accumulators so that the next tile's product runs under this
+// tile's exponentials.
+//
+// A seventeenth warp requests the tiles, issues the products and (pass 2) prepares each query's
+// exponent offset; the other sixteen only read accumulators and do the exponentials.
+// Accumulator: row i of the product is lane i of tensor memory, column j is column j.  A warp can
+// read the 32 lanes of its quadrant (warp % 4), so sixteen warps share a tile as 4 row quadrants
+// x 4 blocks of 32 columns: a thread reads 32 columns of one resident row per tile
+// (tcgen05.ld.32x32b.x32) and keeps that row's running max / sum or column sum over its column
+// blocks; the four partial results of a row are folded through shared memory once, at the end.
+// (One warp per scheduler could not issue the exponentials fast enough: 4 warps took 4900 cycles
+// per tile against 1024 for the exponentials alone.  Staging the tiles with 16-byte cp.async
+// into an unswizzled layout instead of TMA took half of the kernel's time.)
+//
+// Every wait is bounded; a thread that gives up records ZSM_ERR_TIMEOUT and every thread still
+// reaches the end of the kernel, where the tensor memory is released.
 #include "zsm_prefill_full.cuh"
+
+#include <cuda.h>
 
 namespace zsm {
 
 namespace {
 
-constexpr int kFullThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc)
-                 : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void *smem_row) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(smem_u32(smem_row)));
-}
+constexpr int kTcRows = 128;      // resident rows = streamed rows per tile = M = N of one step
+constexpr int kTcEpiThreads = 512;             // 4 row quadrants x 4 column blocks of the accumulator
+constexpr int kTcThreads = kTcEpiThreads + 32;  // + the warp that requests tiles and issues products
+constexpr int kTcStages = 3;      // streamed tiles in shared memory
+constexpr int kTcOffRing = 4;     // per-query exponent offsets, one entry per item in flight
+constexpr int kTcTmemCols = 256;  // two 128-column accumulators
+constexpr int kTcKBlock = 64;     // elements of the head dimension per 128-byte swizzled row
+
+enum : int32_t { WF_MMA = 41, WF_TILE = 42, WF_RESIDENT = 43 };
+
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
+// Shared-memory matrix descriptor of a K-major operand stored as rows of 128 bytes with the
+// 128-byte swizzle (what the tensor map writes): start address in 16-byte units, stride byte
+// offset = 8 rows x 128 bytes, descriptor version 1, layout type 2 (128-byte swizzle).  The
+// leading byte offset is not used for this layout.
+__device__ __forceinline__ uint64_t umma_desc_sw128(const void *smem_ptr) {
+    const uint64_t a = (smem_u32(smem_ptr) >> 4) & 0x3fffu;
+    return a | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ void umma_f16_ss(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t"
+        "}\n"
+        :
+        : "r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                     smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
+          "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+          "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// One box of a 3-D tensor map (head dimension, position, head) into this CTA's shared memory.
+// x is a multiple of 64 elements, so the copy starts on a 128-byte boundary of the row.
+__device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *map, int x, int y, int z,
+                                            uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y),
+        "r"(z)
+        : "memory");
+}
+
+template <int D>
+struct TcSmem {
+    static constexpr int KB = D / kTcKBlock;                 // 128-byte-row blocks per tile
+    static constexpr int KBLOCK = kTcRows * 128;             // bytes of one block: 128 rows x 128 B
+    static constexpr int TILE = KB * KBLOCK;                 // one operand tile
+    static constexpr int a = 0;
+    static constexpr int b = TILE;
+    static constexpr int off = TILE * (1 + kTcStages);
+    static constexpr int comb = off + kTcOffRing * kTcRows * 4;  // [4][128] float2: partial results
+    static constexpr int bars = comb + 4 * kTcRows * 8;          // full[3], mma[2], resident, slot, flag
+    static constexpr int total = bars + 128 + 1024;              // + slack to align the base to 1 KiB
+};
+
 template <typename T, int D, bool COLSUM>
-__global__ void __launch_bounds__(kFullThreads) full_pass_kernel(const FullScoreParams p) {
-    constexpr int STRIDE = D * 2 + 16;  // staged row pitch in bytes: an odd number of 16-byte words
-    constexpr int TILE = kFullBlock * STRIDE;
-    constexpr int KS = D / 16;          // tensor-core steps along the head dimension
-    constexpr int CPR = D * 2 / 16;     // 16-byte chunks per row
-    constexpr int MT = kFullResident / 64;  // 16-row tiles of the resident block per warp
-    extern __shared__ __align__(128) uint8_t smem[];
-    float *off_s = reinterpret_cast<float *>(smem + 2 * TILE);  // [2][64]: pass 2, per query
+__global__ void __launch_bounds__(kTcThreads, 1)
+    full_pass_tc_kernel(const FullScoreParams p, const __grid_constant__ CUtensorMap map_k,
+                        const __grid_constant__ CUtensorMap map_q) {
+    using L = TcSmem<D>;
+    constexpr int KS = D / 16;  // tensor-core steps along the head dimension
+    extern __shared__ uint8_t smem_raw[];
+    // the swizzle pattern repeats every 1024 bytes: tiles start on such a boundary
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    float *off_s = reinterpret_cast<float *>(smem + L::off);
+    float2 *comb = reinterpret_cast<float2 *>(smem + L::comb);
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + L::bars);  // [3] tile landed
+    uint64_t *mma_bar = full_bar + kTcStages;                            // [2] product finished
+    uint64_t *res_bar = mma_bar + 2;                                     // resident block landed
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(res_bar + 1);
+    volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(tmem_slot + 2);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int gq = lane >> 2, tig = lane & 3;
     const int Tn = p.T, G = p.G;
-    const int nb = (Tn + kFullBlock - 1) / kFullBlock;  // streamed tiles that hold a position
-    const int rb = blockIdx.x;                           // the resident block
-    constexpr int RPS = kFullResident / kFullBlock;      // streamed tiles per resident block
+    const int nb = (Tn + kTcRows - 1) / kTcRows;
+    // the longest blocks first: pass 2 walks nb - rb tiles, pass 1 rb + 1
+    const int rb = COLSUM ? blockIdx.x : nb - 1 - blockIdx.x;
     int b, hk, hq = 0;
     if (COLSUM) {
         b = blockIdx.y / p.n_kv_heads;
@@ -66,202 +153,284 @@ __global__ void __launch_bounds__(kFullThreads) full_pass_kernel(const FullScore
         hq = blockIdx.y % (p.n_kv_heads * G);
         hk = hq / G;
     }
-    const T *Kh = static_cast<const T *>(p.K) + ((size_t)b * p.n_kv_heads + hk) * Tn * D;
-    const T *Qb = static_cast<const T *>(p.Q) + (size_t)b * p.n_kv_heads * G * Tn * D;
-    const T *res = COLSUM ? Kh : Qb + (size_t)hq * Tn * D;
+    const int zk = b * p.n_kv_heads + hk;           // head coordinate in the K map
+    const int zq0 = b * p.n_kv_heads * G + hk * G;  // first query head of the group in the Q map
+    const CUtensorMap *map_res = COLSUM ? &map_k : &map_q;
+    const CUtensorMap *map_str = COLSUM ? &map_q : &map_k;
+    const int z_res = COLSUM ? zk : b * p.n_kv_heads * G + hq;
 
-    // resident rows of this thread: gq and gq + 8 of each of the warp's MT 16-row tiles
-    const int rbase = rb * kFullResident + warp * (16 * MT) + gq;
-    uint32_t a[MT][KS][4];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-        const T *r0p = res + (size_t)min(rbase + 16 * mt, Tn - 1) * D;
-        const T *r1p = res + (size_t)min(rbase + 16 * mt + 8, Tn - 1) * D;
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            a[mt][ks][0] = *reinterpret_cast<const uint32_t *>(r0p + 16 * ks + 2 * tig);
-            a[mt][ks][1] = *reinterpret_cast<const uint32_t *>(r1p + 16 * ks + 2 * tig);
-            a[mt][ks][2] = *reinterpret_cast<const uint32_t *>(r0p + 16 * ks + 8 + 2 * tig);
-            a[mt][ks][3] = *reinterpret_cast<const uint32_t *>(r1p + 16 * ks + 8 + 2 * tig);
-        }
-    }
-
-    // streamed tiles: pass 1 key tiles 0 .. the resident block's last row; pass 2 query tiles
-    // from the resident block's first row to the end, for each head of the group
-    const int first = COLSUM ? rb * RPS : 0;
-    const int per = COLSUM ? nb - first : min(rb * RPS + RPS, nb);
+    const int first = COLSUM ? rb : 0;
+    const int per = COLSUM ? nb - rb : rb + 1;
     const int items = COLSUM ? per * G : per;
     const float scale2 = p.scale * kLog2e;
     const float l2lam = log2f(p.lambda);
+    const int quad = warp & 3, cq = warp >> 2;  // accumulator lanes 32 quad.., columns 32 cq..
+    const int rloc = quad * 32 + lane;
+    const int row = rb * kTcRows + rloc;         // the resident row this thread works on
 
-    auto stage_item = [&](int i, int s) {
-        const int g = COLSUM ? i / per : 0;
-        const int jb = first + (COLSUM ? i % per : i);
-        const T *src = COLSUM ? Qb + (size_t)(hk * G + g) * Tn * D : Kh;
-        uint8_t *dst = smem + s * TILE;
-        for (int c = tid; c < kFullBlock * CPR; c += kFullThreads) {
-            const int r = c / CPR, cc = c % CPR;
-            const int grow = min(jb * kFullBlock + r, Tn - 1);
-            cp_async16(dst + r * STRIDE + cc * 16, reinterpret_cast<const uint8_t *>(src + (size_t)grow * D) + cc * 16);
-        }
-        if (COLSUM && tid < kFullBlock) {
-            // exponent offset of query q: decay lambda^(T-1-q) and the row's normaliser
-            const int q = jb * kFullBlock + tid;
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) mbar_init(&full_bar[s], 1);
+        mbar_init(&mma_bar[0], 1);
+        mbar_init(&mma_bar[1], 1);
+        mbar_init(res_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(tmem_slot)),
+                     "r"(kTcTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // exponent offset of query q of head g: decay lambda^(T-1-q) and the row's normaliser
+    // Tile of item i.  Pass 2 walks the query tiles from the last one down: the blocks of a head
+    // start together, so they then ask for the same tiles at about the same time and all but the
+    // first get them from L2.
+    auto tile_of = [&](int i) -> int { return COLSUM ? first + per - 1 - i % per : i; };
+    // (producer warp) the 128 offsets of item i into the ring
+    auto put_offsets = [&](int i) {
+        if (i >= items) return;
+        const float *lse = p.lse + ((size_t)zq0 + i / per) * Tn;
+#pragma unroll
+        for (int k = 0; k < kTcRows / 32; ++k) {
+            const int q = tile_of(i) * kTcRows + k * 32 + lane;
             float o = -INFINITY;
             if (q < Tn) {
-                const float l = p.lse[((size_t)b * p.n_kv_heads * G + hk * G + g) * Tn + q];
                 const float dec = (q == Tn - 1) ? 0.f : static_cast<float>(Tn - 1 - q) * l2lam;
-                o = dec - l * kLog2e;
+                o = dec - lse[q] * kLog2e;
             }
-            off_s[s * kFullBlock + tid] = o;
+            off_s[(i % kTcOffRing) * kTcRows + k * 32 + lane] = o;
         }
-        cp_async_commit();
+    };
+    // (one thread) request item i's tile
+    auto load_item = [&](int i) {
+        if (i >= items) return;
+        const int s = i % kTcStages;
+        const int jb = tile_of(i);
+        const int z = COLSUM ? zq0 + i / per : zk;
+        mbar_arrive_expect_tx(&full_bar[s], L::TILE);
+#pragma unroll
+        for (int kb = 0; kb < L::KB; ++kb)
+            tma_load_3d(smem + L::b + s * L::TILE + kb * L::KBLOCK, map_str, kb * kTcKBlock, jb * kTcRows, z,
+                        &full_bar[s]);
     };
 
-    float m[MT][2], z[MT][2], colsum[MT][2];
+    const bool producer = warp == kTcEpiThreads / 32;
+    if (producer) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(res_bar, L::TILE);
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            m[mt][h] = -INFINITY;  // pass 1: running max / sum (log2 domain)
-            z[mt][h] = 0.f;
-            colsum[mt][h] = 0.f;   // pass 2
+            for (int kb = 0; kb < L::KB; ++kb)
+                tma_load_3d(smem + L::a + kb * L::KBLOCK, map_res, kb * kTcKBlock, rb * kTcRows, z_res, res_bar);
+            for (int i = 0; i < kTcStages; ++i) load_item(i);
         }
-    stage_item(0, 0);
-    for (int i = 0; i < items; ++i) {
-        const int s = i & 1;
-        if (i + 1 < items) {
-            stage_item(i + 1, s ^ 1);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
-        __syncthreads();
-        const int jb = first + (COLSUM ? i % per : i);
-        const uint8_t *tile = smem + s * TILE;
-        // tiles that overlap the resident block's own positions need the causal test
-        const bool diag = jb >= rb * RPS && jb < rb * RPS + RPS;
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {  // half a tile (4 column tiles of 8) at a time
-            float c[MT][4][4];
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                for (int n4 = 0; n4 < 4; ++n4) c[mt][n4][0] = c[mt][n4][1] = c[mt][n4][2] = c[mt][n4][3] = 0.f;
-#pragma unroll
-            for (int n4 = 0; n4 < 4; ++n4) {
-                const int nt = hf * 4 + n4;
-#pragma unroll
-                for (int kq = 0; kq < D / 32; ++kq) {
-                    uint32_t r[4];
-                    ldmatrix_x4(r, tile + (nt * 8 + (lane & 7)) * STRIDE + (kq * 4 + (lane >> 3)) * 16);
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        mma_16x8x16<T>(c[mt][n4], a[mt][2 * kq][0], a[mt][2 * kq][1], a[mt][2 * kq][2],
-                                       a[mt][2 * kq][3], r[0], r[1]);
-                        mma_16x8x16<T>(c[mt][n4], a[mt][2 * kq + 1][0], a[mt][2 * kq + 1][1],
-                                       a[mt][2 * kq + 1][2], a[mt][2 * kq + 1][3], r[2], r[3]);
-                    }
-                }
-            }
-            if (!COLSUM) {
-                // streamed index = key; resident rows = queries; keep key <= query
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    float bm[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-                    for (int n4 = 0; n4 < 4; ++n4) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float v = c[mt][n4][e] * scale2;
-                            if (diag) {
-                                const int key = jb * kFullBlock + (hf * 4 + n4) * 8 + 2 * tig + (e & 1);
-                                if (key > rbase + 16 * mt + 8 * (e >> 1)) v = -INFINITY;
-                            }
-                            c[mt][n4][e] = v;
-                            bm[e >> 1] = fmaxf(bm[e >> 1], v);
-                        }
-                    }
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const float mn = fmaxf(m[mt][h], bm[h]);
-                        const float mu = mn == -INFINITY ? 0.f : mn;
-                        float sum = z[mt][h] * ex2(m[mt][h] - mu);
-#pragma unroll
-                        for (int n4 = 0; n4 < 4; ++n4)
-                            sum += ex2(c[mt][n4][2 * h] - mu) + ex2(c[mt][n4][2 * h + 1] - mu);
-                        z[mt][h] = sum;
-                        m[mt][h] = mn;
-                    }
-                }
-            } else {
-                // streamed index = query; resident rows = keys; keep query >= key
-                const float *off = off_s + s * kFullBlock;
-#pragma unroll
-                for (int n4 = 0; n4 < 4; ++n4) {
-                    const float2 o = *reinterpret_cast<const float2 *>(off + (hf * 4 + n4) * 8 + 2 * tig);
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float v = ex2(fmaf(c[mt][n4][e], scale2, (e & 1) ? o.y : o.x));
-                            if (diag) {
-                                const int q = jb * kFullBlock + (hf * 4 + n4) * 8 + 2 * tig + (e & 1);
-                                if (q < rbase + 16 * mt + 8 * (e >> 1)) v = 0.f;
-                            }
-                            colsum[mt][e >> 1] += v;
-                        }
-                    }
-                }
-            }
-        }
-        __syncthreads();  // the stage is refilled two items from now
+        if (COLSUM)
+            for (int i = 0; i < kTcStages; ++i) put_offsets(i);
     }
 
+    const uint32_t idesc = (1u << 4) | ((Elem<T>::kIsBf16 ? 1u : 0u) << 7) |
+                           ((Elem<T>::kIsBf16 ? 1u : 0u) << 10) | ((kTcRows >> 3) << 17) |
+                           ((kTcRows >> 4) << 24);
+
+    float m = -INFINITY, z = 0.f, colsum = 0.f;
+    bool ok = true;
+    // everything a thread does with the finished product of item j
+    auto epilogue = [&](int j) {
+        const int buf = j & 1;
+        if (!mbar_wait_bounded(&mma_bar[buf], (j >> 1) & 1u, abort_flag, p.status, WF_MMA)) {
+            ok = false;
+            return;
+        }
+        tc_fence_after();
+        const int jb = tile_of(j);
+        const bool diag = jb == rb;
+        const float *off = off_s + (j % kTcOffRing) * kTcRows;
+        uint32_t v[32];
+        tmem_ld32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kTcRows + cq * 32, v);
+        const int col0 = jb * kTcRows + cq * 32;
+        if (!COLSUM) {
+            float bm = -INFINITY;
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
+            for (int e = 0; e < 32; ++e) {
+                float x = __uint_as_float(v[e]) * scale2;
+                if (diag && col0 + e > row) x = -INFINITY;  // keep key <= query
+                v[e] = __float_as_uint(x);
+                bm = fmaxf(bm, x);
+            }
+            const float mn = fmaxf(m, bm);
+            const float mu = mn == -INFINITY ? 0.f : mn;
+            float sum = z * ex2(m - mu);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int row = rbase + 16 * mt + 8 * h;
-            if (!COLSUM) {
-                float mm = m[mt][h], zz = z[mt][h];
+            for (int e = 0; e < 32; ++e) sum += ex2(__uint_as_float(v[e]) - mu);
+            z = sum;
+            m = mn;
+        } else {
 #pragma unroll
-                for (int x = 1; x <= 2; x <<= 1) {
-                    const float mo = __shfl_xor_sync(0xffffffffu, mm, x);
-                    const float zo = __shfl_xor_sync(0xffffffffu, zz, x);
-                    const float mn = fmaxf(mm, mo);
-                    const float mu = mn == -INFINITY ? 0.f : mn;
-                    zz = zz * ex2(mm - mu) + zo * ex2(mo - mu);
-                    mm = mn;
+            for (int e4 = 0; e4 < 8; ++e4) {
+                const float4 o = *reinterpret_cast<const float4 *>(off + cq * 32 + e4 * 4);
+                const float oo[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float x = ex2(fmaf(__uint_as_float(v[e4 * 4 + e]), scale2, oo[e]));
+                    if (diag && col0 + e4 * 4 + e < row) x = 0.f;  // keep query >= key
+                    colsum += x;
                 }
-                if (tig == 0 && row < Tn)
-                    p.lse_out[((size_t)b * p.n_kv_heads * G + hq) * Tn + row] = (mm + log2f(zz)) * kLn2;
-            } else {
-                float v = colsum[mt][h];
-                v += __shfl_xor_sync(0xffffffffu, v, 1);
-                v += __shfl_xor_sync(0xffffffffu, v, 2);
-                if (tig == 0 && row < Tn)
-                    p.scores[((size_t)b * p.n_kv_heads + hk) * Tn + row] = v * (1.0f / static_cast<float>(G));
             }
         }
+    };
+
+    for (int i = 0; i < items; ++i) {
+        tc_fence_before();
+        // every thread has read the accumulator item i will overwrite; leave together on a failure
+        if (__syncthreads_or(!ok)) {
+            ok = false;
+            break;
+        }
+        tc_fence_after();
+        if (producer && lane == 0) {
+            bool ready = i > 0 || mbar_wait_bounded(res_bar, 0, abort_flag, p.status, WF_RESIDENT);
+            ready = ready && mbar_wait_bounded(&full_bar[i % kTcStages], (i / kTcStages) & 1u, abort_flag,
+                                               p.status, WF_TILE);
+            if (ready) {
+                tc_fence_after();
+                const uint8_t *bt = smem + L::b + (i % kTcStages) * L::TILE;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int o = (ks / 4) * L::KBLOCK + (ks % 4) * 32;  // 16 elements = 32 bytes on
+                    umma_f16_ss(tmem_base + (i & 1) * kTcRows, umma_desc_sw128(smem + L::a + o),
+                                umma_desc_sw128(bt + o), idesc, ks > 0);
+                }
+                umma_commit(&mma_bar[i & 1]);
+            } else {
+                ok = false;
+            }
+        }
+        if (producer) {
+            // item i - 1's product frees its stage: request the tile three items on, and its offsets
+            __syncwarp();
+            if (i >= 1) {
+                if (lane == 0 && ok) {
+                    if (mbar_wait_bounded(&mma_bar[(i - 1) & 1], ((i - 1) >> 1) & 1u, abort_flag, p.status, WF_MMA))
+                        load_item(i - 1 + kTcStages);
+                    else
+                        ok = false;
+                }
+                if (COLSUM) put_offsets(i - 1 + kTcStages);
+            }
+        } else if (i >= 1 && ok) {
+            epilogue(i - 1);
+        }
     }
+    tc_fence_before();
+    if (__syncthreads_or(!ok)) ok = false;
+    tc_fence_after();
+    if (ok && items >= 1 && !producer) epilogue(items - 1);
+
+    // fold the four column blocks' partial results of each row
+    if (!producer) comb[cq * kTcRows + rloc] = COLSUM ? make_float2(colsum, 0.f) : make_float2(m, z);
+    tc_fence_before();
+    if (__syncthreads_or(!ok)) ok = false;
+    if (ok && !producer && cq == 0 && row < Tn) {
+        if (!COLSUM) {
+            float mm = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) mm = fmaxf(mm, comb[k * kTcRows + rloc].x);
+            float zz = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 t = comb[k * kTcRows + rloc];
+                zz += t.y * ex2(t.x - mm);  // a block that saw no key has sum 0 and max -inf
+            }
+            p.lse_out[((size_t)b * p.n_kv_heads * G + hq) * Tn + row] = (mm + log2f(zz)) * kLn2;
+        } else {
+            float v = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v += comb[k * kTcRows + rloc].x;
+            p.scores[((size_t)b * p.n_kv_heads + hk) * Tn + row] = v * (1.0f / static_cast<float>(G));
+        }
+    }
+    if (!ok && producer && lane == 0) {
+        // copies that were requested may still land: give them time before the memory goes away
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    __syncwarp();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"(kTcTmemCols)
+                     : "memory");
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link
+// against the driver library directly.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// [heads][T][D] row-major, 16-bit elements, seen as (d, position, head); boxes of 64 x 128 x 1 with
+// the 128-byte swizzle; positions past T read as zero.
+bool make_map(CUtensorMap *map, const void *base, int heads, int T, int D, bool bf16) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t gdim[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)heads};
+    const cuuint64_t gstride[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kTcKBlock, (cuuint32_t)kTcRows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+              const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <typename T, int D>
 int launch_full_one(const FullScoreParams &p, cudaStream_t stream) {
-    constexpr int SMEM = 2 * kFullBlock * (D * 2 + 16) + 2 * kFullBlock * 4;
-    const int nres = (p.T + kFullResident - 1) / kFullResident;
+    constexpr int SMEM = TcSmem<D>::total;
+    CUtensorMap map_k, map_q;
+    if (!make_map(&map_k, p.K, p.batch * p.n_kv_heads, p.T, D, Elem<T>::kIsBf16) ||
+        !make_map(&map_q, p.Q, p.batch * p.n_kv_heads * p.G, p.T, D, Elem<T>::kIsBf16))
+        return static_cast<int>(cudaErrorInvalidValue);
+    const int nres = (p.T + kTcRows - 1) / kTcRows;
     FullScoreParams q = p;
     if (!p.lse) {
         const dim3 grid(nres, p.batch * p.n_kv_heads * p.G);
-        full_pass_kernel<T, D, false><<<grid, kFullThreads, SMEM, stream>>>(q);
+        full_pass_tc_kernel<T, D, false><<<grid, kTcThreads, SMEM, stream>>>(q, map_k, map_q);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return static_cast<int>(e);
         q.lse = p.lse_out;
     }
     const dim3 grid(nres, p.batch * p.n_kv_heads);
-    full_pass_kernel<T, D, true><<<grid, kFullThreads, SMEM, stream>>>(q);
+    full_pass_tc_kernel<T, D, true><<<grid, kTcThreads, SMEM, stream>>>(q, map_k, map_q);
     return static_cast<int>(cudaGetLastError());
+}
+
+template <typename T, int D>
+int prepare_full_one() {
+    cudaError_t e = cudaFuncSetAttribute(full_pass_tc_kernel<T, D, false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::total);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(full_pass_tc_kernel<T, D, true>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::total);
+    return static_cast<int>(e);
 }
 
 }  // namespace
@@ -271,6 +440,14 @@ int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t 
     if (dtype == 1 && D == 128) return launch_full_one<__half, 128>(p, stream);
     if (dtype == 2 && D == 64) return launch_full_one<__nv_bfloat16, 64>(p, stream);
     if (dtype == 2 && D == 128) return launch_full_one<__nv_bfloat16, 128>(p, stream);
+    return -1;
+}
+
+int prepare_full_scores(int dtype, int D) {
+    if (dtype == 1 && D == 64) return prepare_full_one<__half, 64>();
+    if (dtype == 1 && D == 128) return prepare_full_one<__half, 128>();
+    if (dtype == 2 && D == 64) return prepare_full_one<__nv_bfloat16, 64>();
+    if (dtype == 2 && D == 128) return prepare_full_one<__nv_bfloat16, 128>();
     return -1;
 }
 

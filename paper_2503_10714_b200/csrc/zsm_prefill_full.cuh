@@ -6,8 +6,6 @@
 
 namespace zsm {
 
-constexpr int kFullBlock = 64;      // rows of a streamed tile
-constexpr int kFullResident = 128;  // rows of the block a CTA keeps in registers
 
 struct FullScoreParams {
     const void *K;      // [batch][n_kv_heads][T][d]
@@ -15,6 +13,7 @@ struct FullScoreParams {
     const float *lse;   // [batch][n_q_heads][T] natural log-sum-exp of each query's causal row
     float *lse_out;     // same shape, written by the first pass (null when `lse` is supplied)
     float *scores;      // [batch][n_kv_heads][T]
+    int32_t *status;    // sticky device status word of the cache
     int32_t batch, n_kv_heads, G, T;
     float lambda, scale;
 };
@@ -22,5 +21,7 @@ struct FullScoreParams {
 // Enqueues one or both passes on `stream`: row statistics (skipped when p.lse is set), then the
 // decayed column sums.  dtype: 1 fp16, 2 bf16.  Returns a cudaError_t as int; -1: no kernel.
 int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t stream);
+// Raises the kernels' dynamic shared-memory limit; returns a cudaError_t as int (-1: no kernel).
+int prepare_full_scores(int dtype, int D);
 
 }  // namespace zsm
