@@ -12,8 +12,8 @@
 // accumulator in tensor memory, two accumulators so that the next tile's product runs under this
 // tile's exponentials.
 //
-// A seventeenth warp requests the tiles, issues the products and (pass 2) prepares each query's
-// exponent offset; the other sixteen only read accumulators and do the exponentials.
+// A seventeenth warp requests the tiles and issues the products, an eighteenth (pass 2) prepares
+// each query's exponent offset; the other sixteen only read accumulators and do the exponentials.
 // Accumulator: row i of the product is lane i of tensor memory, column j is column j.  A warp can
 // read the 32 lanes of its quadrant (warp % 4), so sixteen warps share a tile as 4 row quadrants
 // x 4 blocks of 32 columns: a thread reads 32 columns of one resident row per tile
@@ -38,7 +38,8 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 constexpr int kTcRows = 128;      // resident rows = streamed rows per tile = M = N of one step
 constexpr int kTcEpiThreads = 512;             // 4 row quadrants x 4 column blocks of the accumulator
-constexpr int kTcThreads = kTcEpiThreads + 32;  // + the warp that requests tiles and issues products
+constexpr int kTcThreads = kTcEpiThreads + 64;  // + a warp that requests tiles and issues products
+                                                // + a warp that prepares the exponent offsets
 constexpr int kTcStages = 3;      // streamed tiles in shared memory
 constexpr int kTcOffRing = 4;     // per-query exponent offsets, one entry per item in flight
 constexpr int kTcTmemCols = 256;  // two 128-column accumulators
@@ -194,19 +195,25 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     // start together, so they then ask for the same tiles at about the same time and all but the
     // first get them from L2.
     auto tile_of = [&](int i) -> int { return COLSUM ? first + per - 1 - i % per : i; };
-    // (producer warp) the 128 offsets of item i into the ring
-    auto put_offsets = [&](int i) {
-        if (i >= items) return;
-        const float *lse = p.lse + ((size_t)zq0 + i / per) * Tn;
+    // (offset warp) the 128 exponent offsets of an item (head g, query tile jb) into ring entry e:
+    // the rows' log-sum-exp are fetched one item ahead of where they are written
+    auto fetch_lse = [&](int g, int jb, float (&l)[kTcRows / 32]) {
 #pragma unroll
         for (int k = 0; k < kTcRows / 32; ++k) {
-            const int q = tile_of(i) * kTcRows + k * 32 + lane;
+            const int q = jb * kTcRows + k * 32 + lane;
+            l[k] = (g < G && q < Tn) ? p.lse[((size_t)zq0 + g) * Tn + q] : 0.f;
+        }
+    };
+    auto put_offsets = [&](int e, int jb, const float (&l)[kTcRows / 32]) {
+#pragma unroll
+        for (int k = 0; k < kTcRows / 32; ++k) {
+            const int q = jb * kTcRows + k * 32 + lane;
             float o = -INFINITY;
             if (q < Tn) {
                 const float dec = (q == Tn - 1) ? 0.f : static_cast<float>(Tn - 1 - q) * l2lam;
-                o = dec - lse[q] * kLog2e;
+                o = dec - l[k] * kLog2e;
             }
-            off_s[(i % kTcOffRing) * kTcRows + k * 32 + lane] = o;
+            off_s[e * kTcRows + k * 32 + lane] = o;
         }
     };
     // (one thread) request item i's tile
@@ -223,6 +230,25 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     };
 
     const bool producer = warp == kTcEpiThreads / 32;
+    const bool offsetter = warp == kTcEpiThreads / 32 + 1;
+    // offset warp: the item whose log-sum-exp it holds (head og, tile ojb, ring entry oe)
+    float lse_ahead[kTcRows / 32] = {0.f, 0.f, 0.f, 0.f};
+    int og = 0, ojb = first + per - 1, oe = 0;
+    auto next_item = [&]() {
+        if (--ojb < first) {
+            ojb = first + per - 1;
+            ++og;
+        }
+        if (++oe == kTcOffRing) oe = 0;
+    };
+    if (offsetter && COLSUM) {
+        for (int i = 0; i < kTcStages; ++i) {
+            fetch_lse(og, ojb, lse_ahead);
+            put_offsets(oe, ojb, lse_ahead);
+            next_item();
+        }
+        fetch_lse(og, ojb, lse_ahead);
+    }
     if (producer) {
         if (lane == 0) {
             mbar_arrive_expect_tx(res_bar, L::TILE);
@@ -231,8 +257,6 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                 tma_load_3d(smem + L::a + kb * L::KBLOCK, map_res, kb * kTcKBlock, rb * kTcRows, z_res, res_bar);
             for (int i = 0; i < kTcStages; ++i) load_item(i);
         }
-        if (COLSUM)
-            for (int i = 0; i < kTcStages; ++i) put_offsets(i);
     }
 
     const uint32_t idesc = (1u << 4) | ((Elem<T>::kIsBf16 ? 1u : 0u) << 7) |
@@ -322,7 +346,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     else
                         ok = false;
                 }
-                if (COLSUM) put_offsets(i - 1 + kTcStages);
+            }
+        } else if (offsetter) {
+            // offsets of the item three on from the one whose exponentials run now
+            if (COLSUM && i >= 1) {
+                put_offsets(oe, ojb, lse_ahead);
+                next_item();
+                fetch_lse(og, ojb, lse_ahead);
             }
         } else if (i >= 1 && ok) {
             epilogue(i - 1);
@@ -331,13 +361,14 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     tc_fence_before();
     if (__syncthreads_or(!ok)) ok = false;
     tc_fence_after();
-    if (ok && items >= 1 && !producer) epilogue(items - 1);
+    const bool epi = warp < kTcEpiThreads / 32;
+    if (ok && items >= 1 && epi) epilogue(items - 1);
 
     // fold the four column blocks' partial results of each row
-    if (!producer) comb[cq * kTcRows + rloc] = COLSUM ? make_float2(colsum, 0.f) : make_float2(m, z);
+    if (epi) comb[cq * kTcRows + rloc] = COLSUM ? make_float2(colsum, 0.f) : make_float2(m, z);
     tc_fence_before();
     if (__syncthreads_or(!ok)) ok = false;
-    if (ok && !producer && cq == 0 && row < Tn) {
+    if (ok && epi && cq == 0 && row < Tn) {
         if (!COLSUM) {
             float mm = -INFINITY;
 #pragma unroll
