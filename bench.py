@@ -353,6 +353,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fullkv", action="store_true",
                     help="skip the uncompressed-cache comparator (same box, same shapes)")
+    ap.add_argument("--no-full-history", action="store_true",
+                    help="skip the full-history (W = T) prompt scoring leg")
     ap.add_argument("--layers", type=int, default=0,
                     help="run a shallower stack than the workload names (profiling captures only; "
                          "the reported config says so)")
@@ -472,7 +474,7 @@ def main():
         fullkv = fullkv_comparator(zb, w, dev, u, stream)
 
     full_hist = None
-    if world == 1 and not args.no_fullkv and w.dtype != "f32":
+    if world == 1 and not args.no_full_history and w.dtype != "f32":
         full_hist = full_history_scores(zb, cache, w, dev, u, stream)
 
     # ---- roofline of the dominant (only) kernel of the timed region ----
