@@ -41,11 +41,11 @@ constexpr int kTcEpiThreads = 512;             // 4 row quadrants x 4 column blo
 constexpr int kTcThreads = kTcEpiThreads + 64;  // + a warp that requests tiles and issues products
                                                 // + a warp that prepares the exponent offsets
 constexpr int kTcStages = 3;      // streamed tiles in shared memory
-constexpr int kTcOffRing = 4;     // per-query exponent offsets, one entry per item in flight
+constexpr int kTcOffRing = 8;     // per-query exponent offsets: entries of the items in flight
 constexpr int kTcTmemCols = 256;  // two 128-column accumulators
 constexpr int kTcKBlock = 64;     // elements of the head dimension per 128-byte swizzled row
 
-enum : int32_t { WF_MMA = 41, WF_TILE = 42, WF_RESIDENT = 43 };
+enum : int32_t { WF_MMA = 41, WF_TILE = 42, WF_RESIDENT = 43, WF_ACC = 44 };
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -137,8 +137,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + L::bars);  // [3] tile landed
     uint64_t *mma_bar = full_bar + kTcStages;                            // [2] product finished
     uint64_t *res_bar = mma_bar + 2;                                     // resident block landed
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(res_bar + 1);
+    uint64_t *acc_free = res_bar + 1;                                    // [2] accumulator read
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_free + 2);
     volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(tmem_slot + 2);
+    // accumulators picked up so far, counted per epilogue warp (paces the offset warp)
+    uint32_t *picked = reinterpret_cast<uint32_t *>(tmem_slot + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Tn = p.T, G = p.G;
@@ -170,10 +173,14 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const int row = rb * kTcRows + rloc;         // the resident row this thread works on
 
     if (tid == 0) {
-        for (int s = 0; s < kTcStages; ++s) mbar_init(&full_bar[s], 1);
+        // a stage is full when its tile has landed and (pass 2) its offsets are written
+        for (int s = 0; s < kTcStages; ++s) mbar_init(&full_bar[s], COLSUM ? 2 : 1);
+        *picked = 0;
         mbar_init(&mma_bar[0], 1);
         mbar_init(&mma_bar[1], 1);
         mbar_init(res_bar, 1);
+        mbar_init(&acc_free[0], kTcEpiThreads / 32);
+        mbar_init(&acc_free[1], kTcEpiThreads / 32);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -242,10 +249,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (++oe == kTcOffRing) oe = 0;
     };
     if (offsetter && COLSUM) {
-        for (int i = 0; i < kTcStages; ++i) {
+        for (int i = 0; i < kTcStages && i < items; ++i) {
             fetch_lse(og, ojb, lse_ahead);
             put_offsets(oe, ojb, lse_ahead);
             next_item();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[i]);
         }
         fetch_lse(og, ojb, lse_ahead);
     }
@@ -278,6 +287,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         const float *off = off_s + (j % kTcOffRing) * kTcRows;
         uint32_t v[32];
         tmem_ld32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kTcRows + cq * 32, v);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(&acc_free[buf]);  // this warp is done with the accumulator
+            if (COLSUM) atomicAdd(picked, 1u);
+        }
         const int col0 = jb * kTcRows + cq * 32;
         if (!COLSUM) {
             float bm = -INFINITY;
@@ -310,19 +325,24 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         }
     };
 
-    for (int i = 0; i < items; ++i) {
-        tc_fence_before();
-        // every thread has read the accumulator item i will overwrite; leave together on a failure
-        if (__syncthreads_or(!ok)) {
-            ok = false;
-            break;
-        }
-        tc_fence_after();
-        if (producer && lane == 0) {
-            bool ready = i > 0 || mbar_wait_bounded(res_bar, 0, abort_flag, p.status, WF_RESIDENT);
-            ready = ready && mbar_wait_bounded(&full_bar[i % kTcStages], (i / kTcStages) & 1u, abort_flag,
-                                               p.status, WF_TILE);
-            if (ready) {
+    // Three roles, tied by mbarriers only (no block-wide barrier per tile):
+    //   mma_bar[b]   producer -> everyone: the product in accumulator b is complete
+    //   acc_free[b]  16 epilogue warps -> producer, offset warp: accumulator b has been read into
+    //                registers (so the exponentials of the item before it are finished too)
+    const bool epi = warp < kTcEpiThreads / 32;
+    if (producer) {
+        if (lane == 0) {
+            for (int i = 0; i < items && ok; ++i) {
+                bool ready = i > 0 || mbar_wait_bounded(res_bar, 0, abort_flag, p.status, WF_RESIDENT);
+                if (i >= 2)  // item i - 2 has left this accumulator
+                    ready = ready && mbar_wait_bounded(&acc_free[i & 1], ((i - 2) >> 1) & 1u, abort_flag,
+                                                       p.status, WF_ACC);
+                ready = ready && mbar_wait_bounded(&full_bar[i % kTcStages], (i / kTcStages) & 1u, abort_flag,
+                                                   p.status, WF_TILE);
+                if (!ready) {
+                    ok = false;
+                    break;
+                }
                 tc_fence_after();
                 const uint8_t *bt = smem + L::b + (i % kTcStages) * L::TILE;
 #pragma unroll
@@ -332,39 +352,46 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                                 umma_desc_sw128(bt + o), idesc, ks > 0);
                 }
                 umma_commit(&mma_bar[i & 1]);
-            } else {
-                ok = false;
-            }
-        }
-        if (producer) {
-            // item i - 1's product frees its stage: request the tile three items on, and its offsets
-            __syncwarp();
-            if (i >= 1) {
-                if (lane == 0 && ok) {
+                if (i >= 1) {
+                    // item i - 1's product frees its stage: request the tile three items on
                     if (mbar_wait_bounded(&mma_bar[(i - 1) & 1], ((i - 1) >> 1) & 1u, abort_flag, p.status, WF_MMA))
                         load_item(i - 1 + kTcStages);
                     else
                         ok = false;
                 }
             }
-        } else if (offsetter) {
-            // offsets of the item three on from the one whose exponentials run now
-            if (COLSUM && i >= 1) {
+        }
+    } else if (offsetter) {
+        if (COLSUM) {
+            // entry of item i + 2, once every epilogue warp has picked up item i - 1 (ring of 8:
+            // the entry's previous owner, item i - 6, was finished long before)
+            for (int i = 1; i + 2 < items && ok; ++i) {
+                // a count, not a barrier phase: the epilogue warps may be two items on by now
+                const uint32_t need = static_cast<uint32_t>(i) * (kTcEpiThreads / 32);
+                const uint64_t t0 = global_timer_ns();
+                while (*reinterpret_cast<volatile uint32_t *>(picked) < need) {
+                    __nanosleep(64);
+                    if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) {
+                        if (!*abort_flag && lane == 0) dev_set_status(p.status, DEV_ERR_TIMEOUT, WF_ACC, blockIdx.x);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                }
+                if (!ok) break;
                 put_offsets(oe, ojb, lse_ahead);
                 next_item();
                 fetch_lse(og, ojb, lse_ahead);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[(i + 2) % kTcStages]);
             }
-        } else if (i >= 1 && ok) {
-            epilogue(i - 1);
         }
+    } else {
+        for (int j = 0; j < items && ok; ++j) epilogue(j);
     }
-    tc_fence_before();
-    if (__syncthreads_or(!ok)) ok = false;
-    tc_fence_after();
-    const bool epi = warp < kTcEpiThreads / 32;
-    if (ok && items >= 1 && epi) epilogue(items - 1);
 
     // fold the four column blocks' partial results of each row
+    __syncwarp();
     if (epi) comb[cq * kTcRows + rloc] = COLSUM ? make_float2(colsum, 0.f) : make_float2(m, z);
     tc_fence_before();
     if (__syncthreads_or(!ok)) ok = false;
