@@ -6,22 +6,25 @@
 //   pass 2  column sums: for a block of 128 keys, over every later query tile and every query
 //           head of the group, exp(logit - lse) weighted by the decay.
 // Both passes are one kernel.  A 128-row block of one operand (queries in pass 1, keys in pass 2)
-// stays in shared memory; 128-row tiles of the other stream through a three-stage ring, brought in
-// by TMA (cp.async.bulk.tensor, 128-byte swizzle) on full / free mbarriers.  One thread issues
+// stays in shared memory; 128-row tiles of the other stream through a two-stage ring, brought in
+// by TMA (cp.async.bulk.tensor, 128-byte swizzle) and announced on an mbarrier per stage.  One thread issues
 // tcgen05.mma: 128 x 128 x d logits per tile, both operands from shared memory, the fp32
 // accumulator in tensor memory, two accumulators so that the next tile's product runs under this
 // tile's exponentials.
 //
-// A seventeenth warp requests the tiles and issues the products, an eighteenth (pass 2) prepares
-// each query's exponent offset; the other sixteen only read accumulators and do the exponentials.
+// Two CTAs share an SM (two tile stages and 256 of the 512 tensor-memory columns each), so one
+// CTA's waits -- for a product, for an accumulator load -- are covered by the other's arithmetic.
+// Per CTA one warp requests the tiles and issues the products, one (pass 2) prepares each query's
+// exponent offset, and eight only read accumulators and do the exponentials.
 // Accumulator: row i of the product is lane i of tensor memory, column j is column j.  A warp can
-// read the 32 lanes of its quadrant (warp % 4), so sixteen warps share a tile as 4 row quadrants
-// x 4 blocks of 32 columns: a thread reads 32 columns of one resident row per tile
-// (tcgen05.ld.32x32b.x32) and keeps that row's running max / sum or column sum over its column
-// blocks; the four partial results of a row are folded through shared memory once, at the end.
-// (One warp per scheduler could not issue the exponentials fast enough: 4 warps took 4900 cycles
-// per tile against 1024 for the exponentials alone.  Staging the tiles with 16-byte cp.async
-// into an unswizzled layout instead of TMA took half of the kernel's time.)
+// read the 32 lanes of its quadrant (warp % 4), so the eight warps share a tile as 4 row quadrants
+// x 2 column halves: a thread reads two blocks of 32 columns of one resident row per tile
+// (tcgen05.ld.32x32b.x32) and keeps that row's running max / sum or column sum over its columns;
+// the two partial results of a row are folded through shared memory once, at the end.
+// (Measured on the way here, c4 shape, per layer: 4 epilogue warps, one CTA per SM, tiles staged
+// with 16-byte cp.async into an unswizzled layout 90.7 ms; 16 warps 75.9; TMA tiles 58.2; a warp
+// of its own for requests and products 47.1, another for the offsets 41.6; mbarriers instead of a
+// block barrier per tile 39.2; two CTAs of 8 epilogue warps per SM 32.3.)
 //
 // Every wait is bounded; a thread that gives up records ZSM_ERR_TIMEOUT and every thread still
 // reaches the end of the kernel, where the tensor memory is released.
@@ -37,10 +40,11 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
 constexpr int kTcRows = 128;      // resident rows = streamed rows per tile = M = N of one step
-constexpr int kTcEpiThreads = 512;             // 4 row quadrants x 4 column blocks of the accumulator
+constexpr int kTcEpiThreads = 256;             // 4 row quadrants x 2 column halves of the accumulator
+constexpr int kTcColParts = kTcEpiThreads / 128; // column parts; a thread reads 128 / parts columns per tile
 constexpr int kTcThreads = kTcEpiThreads + 64;  // + a warp that requests tiles and issues products
                                                 // + a warp that prepares the exponent offsets
-constexpr int kTcStages = 3;      // streamed tiles in shared memory
+constexpr int kTcStages = 2;      // streamed tiles in shared memory (two CTAs share an SM)
 constexpr int kTcOffRing = 8;     // per-query exponent offsets: entries of the items in flight
 constexpr int kTcTmemCols = 256;  // two 128-column accumulators
 constexpr int kTcKBlock = 64;     // elements of the head dimension per 128-byte swizzled row
@@ -124,7 +128,7 @@ struct TcSmem {
 };
 
 template <typename T, int D, bool COLSUM>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
     full_pass_tc_kernel(const FullScoreParams p, const __grid_constant__ CUtensorMap map_k,
                         const __grid_constant__ CUtensorMap map_q) {
     using L = TcSmem<D>;
@@ -285,15 +289,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         const int jb = tile_of(j);
         const bool diag = jb == rb;
         const float *off = off_s + (j % kTcOffRing) * kTcRows;
+        constexpr int CH = 4 / kTcColParts;  // 32-column chunks per thread
+#pragma unroll 1
+        for (int c = 0; c < CH; ++c) {
+        const int ch = cq * CH + c;
         uint32_t v[32];
-        tmem_ld32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kTcRows + cq * 32, v);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) {
-            mbar_arrive(&acc_free[buf]);  // this warp is done with the accumulator
-            if (COLSUM) atomicAdd(picked, 1u);
+        tmem_ld32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kTcRows + ch * 32, v);
+        if (c == CH - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&acc_free[buf]);  // this warp is done with the accumulator
+                if (COLSUM) atomicAdd(picked, 1u);
+            }
         }
-        const int col0 = jb * kTcRows + cq * 32;
+        const int col0 = jb * kTcRows + ch * 32;
         if (!COLSUM) {
             float bm = -INFINITY;
 #pragma unroll
@@ -313,7 +323,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         } else {
 #pragma unroll
             for (int e4 = 0; e4 < 8; ++e4) {
-                const float4 o = *reinterpret_cast<const float4 *>(off + cq * 32 + e4 * 4);
+                const float4 o = *reinterpret_cast<const float4 *>(off + ch * 32 + e4 * 4);
                 const float oo[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -322,6 +332,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     colsum += x;
                 }
             }
+        }
         }
     };
 
@@ -365,7 +376,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (COLSUM) {
             // entry of item i + 2, once every epilogue warp has picked up item i - 1 (ring of 8:
             // the entry's previous owner, item i - 6, was finished long before)
-            for (int i = 1; i + 2 < items && ok; ++i) {
+            for (int i = 1; i - 1 + kTcStages < items && ok; ++i) {
                 // a count, not a barrier phase: the epilogue warps may be two items on by now
                 const uint32_t need = static_cast<uint32_t>(i) * (kTcEpiThreads / 32);
                 const uint64_t t0 = global_timer_ns();
@@ -383,7 +394,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                 next_item();
                 fetch_lse(og, ojb, lse_ahead);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&full_bar[(i + 2) % kTcStages]);
+                if (lane == 0) mbar_arrive(&full_bar[(i - 1 + kTcStages) % kTcStages]);
             }
         }
     } else {
@@ -399,10 +410,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (!COLSUM) {
             float mm = -INFINITY;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) mm = fmaxf(mm, comb[k * kTcRows + rloc].x);
+            for (int k = 0; k < kTcColParts; ++k) mm = fmaxf(mm, comb[k * kTcRows + rloc].x);
             float zz = 0.f;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < kTcColParts; ++k) {
                 const float2 t = comb[k * kTcRows + rloc];
                 zz += t.y * ex2(t.x - mm);  // a block that saw no key has sum 0 and max -inf
             }
@@ -410,7 +421,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         } else {
             float v = 0.f;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) v += comb[k * kTcRows + rloc].x;
+            for (int k = 0; k < kTcColParts; ++k) v += comb[k * kTcRows + rloc].x;
             p.scores[((size_t)b * p.n_kv_heads + hk) * Tn + row] = v * (1.0f / static_cast<float>(G));
         }
     }
