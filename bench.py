@@ -184,7 +184,7 @@ def barrier(world):
 def oracle_sample(w, K, V, Qw, bp, bc, br, steps, layer=0):
     """Times the oracle, as it stands, on one layer's units: state from its own prompt pass
     (untimed), then `steps` decode steps over those units with OpenMP.  Returns
-    (seconds per sampled step, units sampled, threads used)."""
+    (seconds per sampled step, units sampled, threads used, seconds per step on one thread)."""
     from concurrent.futures import ThreadPoolExecutor
 
     from oracle import zsm_oracle as zo
@@ -213,9 +213,16 @@ def oracle_sample(w, K, V, Qw, bp, bc, br, steps, layer=0):
     for step in range(steps):
         _, threads = zo.decode_step_batch(units, qs[step], ks[step], vs[step])
     dt = (time.perf_counter() - t0) / steps
+    # the same units one after another on one thread, a few more steps (inputs reused)
+    n1 = min(steps, 4)
+    t1 = time.perf_counter()
+    for step in range(n1):
+        for i, u in enumerate(units):
+            u.decode_step(qs[step][i], ks[step][i], vs[step][i])
+    dt1 = (time.perf_counter() - t1) / n1
     for u in units:
         u.close()
-    return dt, len(jobs), threads
+    return dt, len(jobs), threads, dt1
 
 
 # ----------------------------------------------------------------------------- per-layer leg
@@ -523,10 +530,11 @@ def main():
         fullkv["compressed_speedup"] = fullkv["ms_per_step"] / ms_per_step
         line["fullkv"] = fullkv
     if world == 1 and not args.no_cpu_baseline and sample_prompt is not None:
-        dt, n_sampled, threads = oracle_sample(w, *sample_prompt, bp, bc, br, args.cpu_steps)
+        dt, n_sampled, threads, dt1 = oracle_sample(w, *sample_prompt, bp, bc, br, args.cpu_steps)
         n_units = w.n_layers * w.batch * w.n_kv_heads
         line["cpu_baseline"] = {
             "value": w.batch / (dt * n_units / n_sampled), "unit": "tokens/s", "cores": threads,
+            "one_thread": w.batch / (dt1 * n_units / n_sampled),
             "kind": "oracle",
             "sample": "%d of %d units (layer 0) x %d decode steps, scaled by units" % (
                 n_sampled, n_units, args.cpu_steps)}
@@ -556,7 +564,7 @@ def main_reference():
     Kp, Vp, Qw = wl.prompt(w, 0)
     K = max(1, min(args.steps, 256))
     W = max(3, args.warmup)
-    dt, n_sampled, threads = oracle_sample(w, Kp, Vp, Qw, bp, bc, br, W + K)
+    dt, n_sampled, threads, dt1 = oracle_sample(w, Kp, Vp, Qw, bp, bc, br, W + K)
     n_units = w.n_layers * w.batch * w.n_kv_heads
     step_s = dt * n_units / n_sampled
     sample = "%d of %d units (layer 0) per step, scaled by units; %d steps" % (n_sampled, n_units, K)
@@ -570,7 +578,7 @@ def main_reference():
                    "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
                    "prompt_len": w.prompt_len, "slots_per_head": int(totals.mean())},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
-                         "sample": sample},
+                         "one_thread": w.batch / (dt1 * n_units / n_sampled), "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0,
                 "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
