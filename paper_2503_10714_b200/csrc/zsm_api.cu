@@ -378,9 +378,11 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
         pl.split = 0;
         if (cfg->tune_split != 1 && cfg->tune_ctas_per_sm == 0 && units * 2 <= c->n_sm) {
             const int limit = cfg->tune_split > 1 ? cfg->tune_split : kSplitMaxCluster;
+            // eight consumer warps: a launch of this form is bound by latencies, not by what its
+            // warps can consume, and the smaller CTA starts sooner (c4 16.9 -> 16.4 us per layer)
             const int warps = cfg->tune_consumer_warps > 0
                                   ? std::min((int)cfg->tune_consumer_warps, kMaxConsumerWarps)
-                                  : kMaxConsumerWarps;
+                                  : kPairConsumerWarps;
             for (int C = kSplitMaxCluster; C >= 2 && pl.split == 0; C >>= 1) {
                 if (C > limit || units * C > c->n_sm) continue;
                 const int ls = split_l_stride(c->cap_max, c->br_max, s.esz, C);
