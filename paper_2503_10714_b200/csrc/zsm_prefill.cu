@@ -1084,6 +1084,7 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
             float n0 = Num[lane];
             float n1 = 1 < nb ? Num[1 * kBlkNS + lane] : 0.f;
             float n2 = 2 < nb ? Num[2 * kBlkNS + lane] : 0.f;
+#pragma unroll 4
             for (int t = 0; t < nb; ++t) {
                 // independent of this token's outcome: its Gram entries with the next three
                 // tokens, and the numerator of the token three ahead
