@@ -304,3 +304,41 @@ def test_cosine_slot_similarity(zb, oracle, split):
     stats = run_decode(zb, oracle, w, np.array([[6, 10]]), np.array([[20, 31]]), np.array([[4, 9]]),
                        steps=220, check_state_every=110, tune_split=split, similarity=1)
     assert stats.merges > 300
+
+
+@pytest.mark.parametrize("split", [0, 1])
+def test_inconsistent_state_is_reported_not_trapped(zb, split):
+    """A full pool whose every token claims to sit inside the proximity window has no eviction
+    candidate.  The kernel records ZSM_ERR_DEVICE_CHECK in the sticky status word, leaves that
+    unit's rows alone (only its token count advances) and keeps running; the healthy unit of
+    the same launch decodes as usual; reading the status clears it."""
+    w = wl.Workload("badstate", 1, 1, 2, 2, 128, "f16", 0, 0, 0, None, 29)
+    cache = GpuCache(zb, w, [[4, 4]], [[4, 4]], [[2, 2]], tune_split=split)
+    try:
+        rs = np.random.RandomState(4)
+        T = 100
+        bad = dict(K=rs.randn(8, 128).astype(np.float32), V=rs.randn(8, 128).astype(np.float32),
+                   score=np.full(8, 0.1, np.float32), pos=np.full(8, T - 1, np.int32),
+                   Kr=rs.randn(2, 128).astype(np.float32), Vr=rs.randn(2, 128).astype(np.float32),
+                   w=np.array([3, 5], np.uint32), n_live=8, n_res=2, T=T)
+        zb.zsm_cache_import_unit(cache.h, 0, 0, 0, 128, bad)
+        q, k, v = (t.cuda() for t in wl.decode_inputs(w, 0))
+        out, vic, slot = cache.decode(q, k, v)
+        assert cache.status() == zb.ZSM_ERR_DEVICE_CHECK
+        assert cache.status() == 0  # sticky until read, then clear
+        assert int(vic.cpu()[0, 0, 0]) == -1 and int(slot.cpu()[0, 0, 0]) == -1
+        after = cache.export(0, 0, 0)
+        np.testing.assert_array_equal(after["pos"], bad["pos"])
+        assert after["n_live"] == 8 and after["n_res"] == 2 and after["T"] == T + 1
+        np.testing.assert_array_equal(after["w"], bad["w"])
+        # the other unit of the launch started empty and took the token
+        ok_unit = cache.export(0, 0, 1)
+        assert ok_unit["n_live"] == 1 and ok_unit["T"] == 1
+        assert torch.isfinite(out.float()).all()
+        # and the cache goes on working
+        cache.decode(q, k, v)
+        assert cache.status() == zb.ZSM_ERR_DEVICE_CHECK  # the bad unit is still bad ...
+        ok_unit = cache.export(0, 0, 1)
+        assert ok_unit["n_live"] == 2 and ok_unit["T"] == 2  # ... the good one is not held up
+    finally:
+        cache.close()
