@@ -925,28 +925,30 @@ size_t merge_warp_smem_bytes() {
 // value to its last bit), so D0 is an fp32-accumulated product of exact operands.
 // ---------------------------------------------------------------------------
 constexpr int kBlkTokens = 64;
-constexpr int kBlkNS = 33;              // row stride of the numerator table (bank-conflict free)
 constexpr int kBlkGS = kBlkTokens + 4;  // row stride of the Gram matrix
 
-template <int D>
+template <int D, int NS>
 struct BlkSmem {
     static constexpr int ROWB = D * 2;
     static constexpr size_t tokK = 0;                                        // [2][64][ROWB]
     static constexpr size_t tokV = tokK + 2 * kBlkTokens * ROWB;             // [2][64][ROWB]
-    static constexpr size_t krm = tokV + 2 * kBlkTokens * ROWB;              // [32][D] fp32
-    static constexpr size_t vrm = krm + 32 * D * 4;                          // [32][D] fp32
-    static constexpr size_t krs = vrm + 32 * D * 4;                          // [3][32][D] 16-bit
-    static constexpr size_t num = krs + 3 * 32 * ROWB;                       // [64][33] fp32
-    static constexpr size_t gm = num + kBlkTokens * kBlkNS * 4;              // [64][68] fp32
+    static constexpr size_t krm = tokV + 2 * kBlkTokens * ROWB;              // [NS][D] fp32
+    static constexpr size_t vrm = krm + NS * D * 4;                          // [NS][D] fp32
+    static constexpr size_t krs = vrm + NS * D * 4;                          // [3][NS][D] 16-bit
+    static constexpr size_t num = krs + 3 * NS * ROWB;                       // [64][NS + 1] fp32
+    static constexpr size_t gm = num + kBlkTokens * (NS + 1) * 4;            // [64][68] fp32
     static constexpr size_t tgt = gm + kBlkTokens * kBlkGS * 4;              // [64] int
-    static constexpr size_t wc = tgt + kBlkTokens * 4;                       // [32] fp32 counts
-    static constexpr size_t total = wc + 32 * 4;
+    static constexpr size_t wc = tgt + kBlkTokens * 4;                       // [NS] fp32 counts
+    static constexpr size_t total = wc + NS * 4;
 };
 
-template <typename T, int D>
+template <typename T, int D, int NS>
 __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const PrefillParams p) {
     using E = Elem<T>;
-    using SM = BlkSmem<D>;
+    using SM = BlkSmem<D, NS>;
+    constexpr int NS1 = NS + 1;   // row stride of the numerator table (bank-conflict free)
+    constexpr int SPL = NS / 32;  // merged slots a lane of the chain warp watches
+    constexpr int NTD = NS / 8;   // 8-slot column tiles of the numerator table
     static_assert(sizeof(T) == 2, "16-bit storage");
     constexpr int ROWB = D * 2;
     constexpr int CPR = ROWB / 16;
@@ -991,13 +993,13 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
         const T m = E::from_float(r1);
         const T l = E::from_float(r1 - E::to_float(m));
         s0[0] = h;
-        s0[32 * D] = m;
-        s0[2 * 32 * D] = l;
+        s0[NS * D] = m;
+        s0[2 * NS * D] = l;
     };
 
     // ---- fill: the first B_r evicted tokens take the free slots as they are (Alg. 1) ----
     const int n_fill = min(Br, n_ev);
-    for (int k = tid; k < 32 * D; k += blockDim.x) {
+    for (int k = tid; k < NS * D; k += blockDim.x) {
         const int r = k / D, e = k % D;
         float kv = 0.f, vv = 0.f;
         if (r < n_fill) {
@@ -1009,7 +1011,7 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
         VrM[k] = vv;
         write_split(r, e, kv);
     }
-    if (tid < 32) wc[tid] = tid < n_fill ? 1.f : 0.f;
+    if (tid < NS) wc[tid] = tid < n_fill ? 1.f : 0.f;
     if (targets)
         for (int i = tid; i < n_fill; i += blockDim.x) targets[i] = -2;
 
@@ -1039,16 +1041,16 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
         const uint8_t *bV = tokV + (size_t)buf * NB * ROWB;
 
         // ---- bulk: D0 (16 tiles of 16 tokens x 8 slots) and Gm (32 tiles of 16 x 8 tokens) ----
-        for (int item = warp; item < 48; item += n_warps) {
-            const bool is_g = item >= 16;
-            const int it = is_g ? item - 16 : item;
-            const int mt = is_g ? it / 8 : it / 4, nt = is_g ? it % 8 : it % 4;
+        for (int item = warp; item < 4 * NTD + 32; item += n_warps) {
+            const bool is_g = item >= 4 * NTD;
+            const int it = is_g ? item - 4 * NTD : item;
+            const int mt = is_g ? it / 8 : it / NTD, nt = is_g ? it % 8 : it % NTD;
             if (!is_g && nt * 8 >= Br) continue;
             const uint8_t *pa = bK + (mt * 16 + gq) * ROWB + tig * 16;
             float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
             const int n_split = is_g ? 1 : 3;
             for (int sp = 0; sp < n_split; ++sp) {
-                const uint8_t *pb = (is_g ? bK : KrS + (size_t)sp * 32 * ROWB) + (nt * 8 + gq) * ROWB + tig * 16;
+                const uint8_t *pb = (is_g ? bK : KrS + (size_t)sp * NS * ROWB) + (nt * 8 + gq) * ROWB + tig * 16;
 #pragma unroll
                 for (int j = 0; j < SEG; ++j) {
                     const uint4 ra = *reinterpret_cast<const uint4 *>(pa + j * 64);
@@ -1066,10 +1068,10 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
                 Gm[(row + 8) * kBlkGS + col + 1] = c0[3] + c1[3];
             } else {
                 const float w0a = wc[col], w0b = wc[col + 1];
-                Num[row * kBlkNS + col] = w0a * (c0[0] + c1[0]);
-                Num[row * kBlkNS + col + 1] = w0b * (c0[1] + c1[1]);
-                Num[(row + 8) * kBlkNS + col] = w0a * (c0[2] + c1[2]);
-                Num[(row + 8) * kBlkNS + col + 1] = w0b * (c0[3] + c1[3]);
+                Num[row * NS1 + col] = w0a * (c0[0] + c1[0]);
+                Num[row * NS1 + col + 1] = w0b * (c0[1] + c1[1]);
+                Num[(row + 8) * NS1 + col] = w0a * (c0[2] + c1[2]);
+                Num[(row + 8) * NS1 + col + 1] = w0b * (c0[3] + c1[3]);
             }
         }
         __syncthreads();
@@ -1079,37 +1081,61 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
         // their corrections there; shared memory is corrected only from four tokens ahead, so
         // no shared-memory round trip sits between one token's argmax and the next.
         if (warp == 0) {
-            float w = lane < Br ? wc[lane] : 1.f;
-            float rw = __frcp_rn(w), rw_next = __frcp_rn(w + 1.f);
-            float n0 = Num[lane];
-            float n1 = 1 < nb ? Num[1 * kBlkNS + lane] : 0.f;
-            float n2 = 2 < nb ? Num[2 * kBlkNS + lane] : 0.f;
+            // lane l watches slots l, l + 32, ..
+            float w[SPL], rw[SPL], rwn[SPL], n0[SPL], n1[SPL], n2[SPL];
+#pragma unroll
+            for (int s = 0; s < SPL; ++s) {
+                const int slot = lane + 32 * s;
+                w[s] = slot < Br ? wc[slot] : 1.f;
+                rw[s] = __frcp_rn(w[s]);
+                rwn[s] = __frcp_rn(w[s] + 1.f);
+                n0[s] = Num[slot];
+                n1[s] = 1 < nb ? Num[1 * NS1 + slot] : 0.f;
+                n2[s] = 2 < nb ? Num[2 * NS1 + slot] : 0.f;
+            }
 #pragma unroll 4
             for (int t = 0; t < nb; ++t) {
                 // independent of this token's outcome: its Gram entries with the next three
-                // tokens, and the numerator of the token three ahead
+                // tokens, and the numerators of the token three ahead
                 const float g1 = t + 1 < nb ? Gm[t * kBlkGS + t + 1] : 0.f;
                 const float g2 = t + 2 < nb ? Gm[t * kBlkGS + t + 2] : 0.f;
                 const float g3 = t + 3 < nb ? Gm[t * kBlkGS + t + 3] : 0.f;
-                float n3 = t + 3 < nb ? Num[(t + 3) * kBlkNS + lane] : 0.f;
-                const float val = n0 * rw;  // k_r . k_t  (Eq. (hatr))
-                const uint32_t key = lane < Br ? order_key(val) : 0u;
-                const uint32_t best = __reduce_max_sync(0xffffffffu, key);
-                const int rhat = __ffs(__ballot_sync(0xffffffffu, key == best && lane < Br)) - 1;
-                const bool me = lane == rhat;
+                float n3[SPL];
+                uint32_t key[SPL], kmax = 0u;
+#pragma unroll
+                for (int s = 0; s < SPL; ++s) {
+                    const int slot = lane + 32 * s;
+                    n3[s] = t + 3 < nb ? Num[(t + 3) * NS1 + slot] : 0.f;
+                    key[s] = slot < Br ? order_key(n0[s] * rw[s]) : 0u;  // k_r . k_t  (Eq. (hatr))
+                    kmax = key[s] > kmax ? key[s] : kmax;
+                }
+                const uint32_t best = __reduce_max_sync(0xffffffffu, kmax);
+                int rhat = -1;  // equal values go to the lowest slot: slots l before slots l + 32
+#pragma unroll
+                for (int s = 0; s < SPL; ++s) {
+                    const unsigned bal = __ballot_sync(0xffffffffu, key[s] == best && lane + 32 * s < Br);
+                    if (rhat < 0 && bal) rhat = 32 * s + __ffs(bal) - 1;
+                }
                 if (lane == 0) tgt[t] = rhat;
-                w += me ? 1.f : 0.f;
-                rw = me ? rw_next : rw;
-                rw_next = __frcp_rn(w + 1.f);
-                n1 += me ? g1 : 0.f;
-                n2 += me ? g2 : 0.f;
-                n3 += me ? g3 : 0.f;
+#pragma unroll
+                for (int s = 0; s < SPL; ++s) {
+                    const bool me = lane + 32 * s == rhat;
+                    w[s] += me ? 1.f : 0.f;
+                    rw[s] = me ? rwn[s] : rw[s];
+                    rwn[s] = __frcp_rn(w[s] + 1.f);
+                    n1[s] += me ? g1 : 0.f;
+                    n2[s] += me ? g2 : 0.f;
+                    n3[s] += me ? g3 : 0.f;
+                }
                 for (int u = t + 4 + lane; u < nb; u += 32)
-                    Num[u * kBlkNS + rhat] += Gm[t * kBlkGS + u];  // Gm is symmetric: row t
+                    Num[u * NS1 + rhat] += Gm[t * kBlkGS + u];  // Gm is symmetric: row t
                 __syncwarp();
-                n0 = n1;
-                n1 = n2;
-                n2 = n3;
+#pragma unroll
+                for (int s = 0; s < SPL; ++s) {
+                    n0[s] = n1[s];
+                    n1[s] = n2[s];
+                    n2[s] = n3[s];
+                }
             }
         }
         __syncthreads();
@@ -1167,7 +1193,7 @@ __global__ void __launch_bounds__(1024) prefill_merge_blocked_kernel(const Prefi
         Kr_g[k] = KrM[k];
         Vr_g[k] = VrM[k];
     }
-    if (tid < n_res) w_g[tid] = static_cast<uint32_t>(wc[tid]);
+    for (int k = tid; k < n_res; k += blockDim.x) w_g[k] = static_cast<uint32_t>(wc[k]);
 }
 
 // ---------------------------------------------------------------------------
@@ -1242,7 +1268,10 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
         prefill_merge_warp_kernel<T, D><<<p.units, 32, merge_warp_smem_bytes<T, D>(), stream>>>(p);
     else if (max_br <= 32 && sizeof(T) == 2) {
         if constexpr (sizeof(T) == 2)
-            prefill_merge_blocked_kernel<T, D><<<p.units, 1024, BlkSmem<D>::total, stream>>>(p);
+            prefill_merge_blocked_kernel<T, D, 32><<<p.units, 1024, BlkSmem<D, 32>::total, stream>>>(p);
+    } else if (max_br <= 64 && sizeof(T) == 2 && p.units <= 2 * p.n_sm) {
+        if constexpr (sizeof(T) == 2)
+            prefill_merge_blocked_kernel<T, D, 64><<<p.units, 1024, BlkSmem<D, 64>::total, stream>>>(p);
     } else if (max_br <= 32)
         prefill_merge_rows_kernel<T, D, 1><<<p.units, kRowMergeThreads, merge_rows_smem_bytes<T, D>(), stream>>>(p);
     else if (max_br <= 64)
@@ -1275,8 +1304,11 @@ int prepare_all() {
                              (int)merge_smem_bytes<D>(prefill_max_residual(D), D * (int)sizeof(T)));
     if (e != cudaSuccess) return static_cast<int>(e);
     if constexpr (sizeof(T) == 2) {
-        e = cudaFuncSetAttribute(prefill_merge_blocked_kernel<T, D>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BlkSmem<D>::total);
+        e = cudaFuncSetAttribute(prefill_merge_blocked_kernel<T, D, 32>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BlkSmem<D, 32>::total);
+        if (e != cudaSuccess) return static_cast<int>(e);
+        e = cudaFuncSetAttribute(prefill_merge_blocked_kernel<T, D, 64>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BlkSmem<D, 64>::total);
         if (e != cudaSuccess) return static_cast<int>(e);
     }
     e = cudaFuncSetAttribute(prefill_merge_warp_kernel<T, D>,
