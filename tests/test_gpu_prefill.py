@@ -82,9 +82,9 @@ def test_prompt_pass_degenerate_budgets(zb, oracle, budgets):
 
 @pytest.mark.parametrize("br", [3, 33, 100, 150])
 def test_residual_pool_sizes(zb, oracle, br):
-    """Residual pools on both sides of the sizes at which the merge kernel changes form: merged
-    keys in registers with one, two or four rows per thread (B_r <= 32, 64, 128), in shared
-    memory beyond that."""
+    """Residual pools on both sides of the sizes at which the merge kernel changes form: the
+    blocked form with one or two slots per lane of its chain warp (B_r <= 32, 64), merged keys
+    in registers with four rows per thread (B_r <= 128), in shared memory beyond that."""
     w = wl.Workload("pool", 1, 1, 2, 2, 128, "f16", 1500, 0, 16, None, 25)
     cache = GpuCache(zb, w, [[40, 64]], [[60, 90]], [[br, max(1, br // 2)]])
     stats = ParityStats()
