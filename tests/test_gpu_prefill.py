@@ -181,3 +181,16 @@ def test_prompt_pass_cosine_slot_similarity(zb, oracle, br):
         assert cache.status() == 0 and stats.merges > 1000
     finally:
         cache.close()
+
+
+def test_residual_pool_of_two_rows_per_thread_fp32(zb, oracle):
+    """fp32 storage has no blocked form: 33..64 merged slots run the register form with two rows
+    per thread."""
+    w = wl.Workload("pool32", 1, 1, 2, 2, 64, "f32", 900, 0, 16, None, 30)
+    cache = GpuCache(zb, w, [[30, 40]], [[40, 50]], [[40, 64]])
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats)
+        assert cache.status() == 0 and stats.merges > 1200
+    finally:
+        cache.close()
