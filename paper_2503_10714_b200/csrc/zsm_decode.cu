@@ -116,7 +116,9 @@ __device__ __forceinline__ void load4(const T *p, float (&f)[4]) {
 // WIDE: up to sixteen consumer warps in one CTA per SM, for launches with no more units than
 // SMs, where a CTA has an SM to itself and its speed is what its warps can consume; otherwise
 // up to eight consumer warps and two CTAs per SM.  Same code: the warp count is the launch's.
-template <typename T, int D, int G, bool WIDE>
+// COS: the cosine option of Eq. (hatr), compiled into its own instantiation (as a run-time branch
+// it cost the default kernel registers: the G = 4 kernel began to spill).
+template <typename T, int D, int G, bool WIDE, bool COS>
 __global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 2)
     decode_fused_kernel(const DecodeParams p) {
     using E = Elem<T>;
@@ -358,7 +360,7 @@ __global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 
                     // Eq. (hatr): raw dot product with every merged key (or its cosine form);
                     // ties to the lowest slot
                     float nt2 = 0.f;
-                    if (p.cosine) {
+                    if constexpr (COS) {
                         nt2 = kc[0] * kc[0];
                         nt2 = fmaf(kc[1], kc[1], nt2);
                         nt2 = fmaf(kc[2], kc[2], nt2);
@@ -384,7 +386,7 @@ __global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 
                             acc = fmaf(kr[u].z, kc[2], acc);
                             acc = fmaf(kr[u].w, kc[3], acc);
                             acc = group_sum<LPR32>(acc);
-                            if (p.cosine) {
+                            if constexpr (COS) {
                                 float nr2 = kr[u].x * kr[u].x;
                                 nr2 = fmaf(kr[u].y, kr[u].y, nr2);
                                 nr2 = fmaf(kr[u].z, kr[u].z, nr2);
@@ -966,27 +968,40 @@ int launch_one(const DecodeParams &p, int grid, int consumer_warps, bool wide, c
     const int threads = (consumer_warps + kExtraWarps) * 32;
     const DecodeSmem L = decode_smem_layout(p.stages, G, D, D * (int)sizeof(T), p.l_stride,
                                             p.br_max_pad, consumer_warps);
-    if (wide)
-        decode_fused_kernel<T, D, G, true><<<grid, threads, L.total, stream>>>(p);
-    else
-        decode_fused_kernel<T, D, G, false><<<grid, threads, L.total, stream>>>(p);
+    if (wide) {
+        if (p.cosine)
+            decode_fused_kernel<T, D, G, true, true><<<grid, threads, L.total, stream>>>(p);
+        else
+            decode_fused_kernel<T, D, G, true, false><<<grid, threads, L.total, stream>>>(p);
+    } else {
+        if (p.cosine)
+            decode_fused_kernel<T, D, G, false, true><<<grid, threads, L.total, stream>>>(p);
+        else
+            decode_fused_kernel<T, D, G, false, false><<<grid, threads, L.total, stream>>>(p);
+    }
     return static_cast<int>(cudaGetLastError());
 }
 
 template <typename T, int D, int G>
 int prepare_one(int smem_bytes, int threads, int *max_ctas) {
-    cudaError_t ew = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, true>,
+    cudaError_t ew = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, true, false>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           kMaxDynamicSmem);
+    if (ew == cudaSuccess)
+        ew = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, true, true>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+    if (ew == cudaSuccess)
+        ew = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, false, true>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
     if (ew != cudaSuccess) return static_cast<int>(ew);
     // The limit belongs to the kernel, not to a cache: caches of one shape but different budgets
     // ask for different amounts, so it is raised to the most any of them can ask for.
-    cudaError_t e = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, false>,
+    cudaError_t e = cudaFuncSetAttribute(decode_fused_kernel<T, D, G, false, false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kMaxDynamicSmem);
     if (e != cudaSuccess) return static_cast<int>(e);
     int n = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_fused_kernel<T, D, G, false>, threads,
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_fused_kernel<T, D, G, false, false>, threads,
                                                       smem_bytes);
     if (max_ctas) *max_ctas = n;
     return static_cast<int>(e);
