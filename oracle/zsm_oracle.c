@@ -471,6 +471,7 @@ int zso_prefill_compress(zso_unit *u, const double *K, const double *V, const do
         if (targets_out) targets_out[ie] = slot;
         R.n_near_tie_merge += nt;
         R.n_mismatch_merge += mm;
+        R.n_exact_tie_merge += et;
         if (gap < R.min_merge_gap) R.min_merge_gap = gap;
         ie += 1;
     }

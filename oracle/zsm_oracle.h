@@ -23,7 +23,9 @@
  * merge conservation laws; occupancy bounds; brute-force score recomputation;
  * an independently written single-pool formulation; restriction-to-retained
  * equivalence for B_r = 0; naive causal-attention scores for the prompt pass;
- * brute-force sort for the prompt selection.
+ * brute-force sort for the prompt selection; constructed exact ties of the
+ * residual arg-max (identical slots, equal products) in both the decode step
+ * and the prompt chain; the two ratios of the budget split.
  * Parity unpinned (no published worked example or code to compare with): the
  * order in which the prompt's evicted tokens are merged, the default score
  * window, and the rounding of the budget split helper.
@@ -87,6 +89,8 @@ typedef struct {
     int32_t n_mismatch_merge;
     double min_merge_gap;
     double sel_gap;        /* (smallest kept score - largest evicted score)/largest evicted */
+    int32_t n_exact_tie_merge; /* hinted merge targets that differed from the oracle's own although
+                                * the two fp32 dot products were equal (tie-rule breaches) */
 } zso_prefill_report;
 
 zso_unit *zso_unit_new(const zso_params *p);

@@ -61,7 +61,7 @@ class PrefillReport(C.Structure):
     _fields_ = [("n_evicted", C.c_int32), ("n_near_tie_sel", C.c_int32),
                 ("n_mismatch_sel", C.c_int32), ("n_near_tie_merge", C.c_int32),
                 ("n_mismatch_merge", C.c_int32), ("min_merge_gap", C.c_double),
-                ("sel_gap", C.c_double)]
+                ("sel_gap", C.c_double), ("n_exact_tie_merge", C.c_int32)]
 
 
 _lib = None

@@ -206,11 +206,14 @@ def prefill_check(oracle, cache: GpuCache, layer, b, h, K, V, Qw, dbg, stats: Pa
     assert r.n_mismatch_sel == 0, f"{tag}: eviction sets differ beyond near ties (gap {r.sel_gap:.3e})"
     assert r.n_mismatch_merge == 0, f"{tag}: merge targets differ beyond near ties (min gap {r.min_merge_gap:.3e})"
     assert r.n_evicted == n_ev, f"{tag}: evicted {n_ev} vs oracle {r.n_evicted}"
+    assert r.n_exact_tie_merge == 0, (f"{tag}: {r.n_exact_tie_merge} merge targets were not the lowest "
+                                      "slot among exactly equal dot products")
     np.testing.assert_array_equal(res.evicted, ev_gpu, err_msg=f"{tag}: eviction flags")
     np.testing.assert_array_equal(res.targets, tg_gpu, err_msg=f"{tag}: merge targets")
     stats.selections += n_ev
     stats.merges += int((tg_gpu >= 0).sum())
     stats.victim_near_ties += r.n_near_tie_sel
     stats.merge_near_ties += r.n_near_tie_merge
+    stats.exact_tie_breaches += r.n_exact_tie_merge
     state_check(unit, cache.export(layer, b, h), stats, tag=tag + " state after prompt pass")
     return unit

@@ -123,27 +123,6 @@ def test_budget_at_least_context_is_full_attention(zb):
         cache.close()
 
 
-def test_exact_ties_resolve_by_position(zb):
-    """Bit-identical tokens give bit-identical scores on the GPU too: the evicted one must be
-    the lowest position among the minima (lam = 0, as in the oracle's pin)."""
-    w = wl.Workload("ties", 1, 1, 1, 1, 64, "f32", 0, 0, 0, None, 14)
-    cache = GpuCache(zb, w, [[1]], [[2]], [[0]], lam=0.0)
-    try:
-        def tok(x):
-            t = torch.zeros(1, 1, 1, 64)
-            t[..., 0] = x
-            return t.cuda()
-        q, ones = tok(1.0), torch.ones(1, 1, 1, 64).cuda()
-        seq = [1.0, 1.0, 5.0, 5.0, 5.0]
-        victims = []
-        for x in seq:
-            _, vic, _ = cache.decode(q, tok(x), ones)
-            victims.append(int(vic.cpu()[0, 0, 0]))
-        assert victims == [-1, -1, -1, 0, 1]
-    finally:
-        cache.close()
-
-
 def test_decode_from_imported_large_state(zb, oracle):
     """A unit larger than one (score, pos) tile (2048 entries) and a residual pool of 60
     slots: state built by the oracle's prompt pass, imported through the C ABI, then decoded

@@ -334,6 +334,62 @@ def test_merge_target_is_max_raw_dot_product(oracle):
     assert w.tolist()[0] == 2
 
 
+@pytest.mark.parametrize("kind", ["identical", "equal_dot"])
+def test_merge_tie_goes_to_lowest_slot(oracle, kind):
+    """Eq. (hatr) with two slots that give the evicted token exactly the same dot product --
+    bit-identical keys, or different keys whose products happen to agree: the lowest slot
+    takes the token (small integers: every product and sum is exact)."""
+    d = 4
+    u = oracle.Unit(d, 1, Bp=1, Bc=1, Br=2, lam=0.0)
+    q = np.array([[0.0, 0, 0, 1.0]])
+    vv = np.arange(d, dtype=np.float64)
+    second = [2.0, 0, 0, -40] if kind == "identical" else [0.0, 2.0, 0, -40]
+    toks = [np.array([2.0, 0, 0, -40]),       # pos 0 -> residual slot 0
+            np.array(second),                 # pos 1 -> residual slot 1
+            np.array([1.0, 1.0, 0, -36]),     # pos 2: dot 1442 with slot 0 and with slot 1
+            np.array([0.0, 0, 0, 20]), np.array([0.0, 0, 0, 20])]
+    reps = [u.decode_step(q, k, vv * (i + 1))[1] for i, k in enumerate(toks)]
+    seq = [(r.victim_pos, r.merge_slot) for r in reps]
+    assert seq == [(-1, -1), (-1, -1), (0, -2), (1, -2), (2, 0)]
+    assert reps[4].merge_runner_slot == 1 and reps[4].merge_gap == 0.0
+    Kr, Vr, w = u.residual()
+    assert w.tolist() == [2, 1]
+    np.testing.assert_array_equal(Kr[0], (toks[0] + toks[2]) / 2)
+    np.testing.assert_array_equal(Kr[1], toks[1])
+    np.testing.assert_array_equal(Vr[0], (vv * 1 + vv * 3) / 2)
+
+
+@pytest.mark.parametrize("Br", [2, 9, 40])
+def test_planted_merge_ties_in_a_decode_stream(oracle, Br):
+    """The planted-tie construction of tie_streams (pairs of slots front / back of the pool,
+    identical keys or equal products, then tokens that tie between them) driven through the
+    decode step: with lam = 1 and imported scores spaced far apart the victims come out in a
+    known order, and each tie token must go to the lower slot of its pair."""
+    from tie_streams import planted_prompt, tie_tokens
+    d, Bp, Bc = 16, 10, 12     # B_p > number of steps: no decoded token leaves proximity
+    rng = np.random.default_rng(40 + Br)
+    ties, want = tie_tokens(Br, d)
+    # prompt: the B_r slot fillers are evicted (they fill the slots); the tie tokens are kept
+    # with the lowest scores, in order, so that decoding evicts them one per step
+    K, V, s, n_ev, _ = planted_prompt(rng, d, Bp, Bc, Br, n_more=0)
+    n_tie = len(want)
+    assert 2 <= n_tie < Bp
+    s[Br:Br + n_tie] = 10.0 * (1 + np.arange(n_tie))       # kept, evicted first later on
+    s[Br + n_tie:] = 1000.0 + 10.0 * np.arange(len(s) - Br - n_tie)
+    s[:Br] = 0.25
+    u = oracle.Unit(d, 1, Bp, Bc + n_tie, Br, lam=1.0)
+    res = u.prefill_compress(K, V, scores=s)
+    assert np.flatnonzero(res.evicted).tolist() == list(range(Br)) and set(res.targets) == {-2}
+    got = []
+    for t in range(n_tie):
+        q = rng.normal(size=(1, d))
+        _, rep = u.decode_step(q, rng.normal(size=d), rng.normal(size=d))
+        assert rep.victim_pos == Br + t
+        assert rep.merge_gap == 0.0
+        got.append(rep.merge_slot)
+    assert got == want
+
+
 def test_cosine_form_prefers_the_aligned_slot(oracle):
     """The cosine form of Eq. (hatr) (commented out beside it in the paper's source): on the
     same stream as above the better aligned short slot wins, and every merge target of a
@@ -427,3 +483,19 @@ def test_budget_split_golden(oracle):
         assert oracle.split_budget(B) == (bp, bc, br)
         assert bp + bc + br == B
     assert oracle.split_budget(100, 0.5, 0.0) == (50, 50, 0)
+
+
+def test_budget_split_holds_the_two_ratios(oracle):
+    """App. C.2 fixes two ratios: B_p / B (0.5 recommended) and B_r / (B - B_p) (0.02).  However
+    the helper rounds, an integer split can be held to them: B_p within one slot of 0.5 B,
+    B_r within half a slot of 0.02 (B - B_p) or at its floor of one slot, B_c the remainder."""
+    for B in list(range(1, 3000)) + list(range(3000, 60001, 37)) + [60000]:
+        bp, bc, br = oracle.split_budget(B)
+        assert bp + bc + br == B and min(bp, bc, br) >= 0 and bp + bc >= 1
+        assert abs(bp - 0.5 * B) < 1.0
+        assert abs(br - 0.02 * (B - bp)) <= 0.5 or br == 1 or (br == 0 and B == 1)
+    for tail, dense in [(0.3, 0.05), (0.7, 0.1), (0.5, 0.2), (0.1, 0.01)]:
+        for B in (64, 205, 819, 2700, 10800, 54000):
+            bp, bc, br = oracle.split_budget(B, tail, dense)
+            assert bp + bc + br == B and abs(bp - tail * B) < 1.0
+            assert abs(br - dense * (B - bp)) <= 0.5 or br == 1

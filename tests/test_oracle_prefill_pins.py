@@ -184,3 +184,22 @@ def test_prefill_hints(oracle):
     bad[-1] = 1 - bad[-1]
     r = u3.prefill_compress(K, V, scores=s, hint_targets=bad, tol=1e-9)
     assert r.report.n_mismatch_merge == 1 and r.targets.tolist() == own3.targets.tolist()
+
+
+@pytest.mark.parametrize("Br", [2, 9, 40])
+def test_planted_merge_ties_in_the_prompt_chain(oracle, Br):
+    """Exact ties of Eq. (hatr) planted in the prompt's evicted stream (tie_streams): each
+    tie token goes to the lower slot of its pair, and the whole chain equals the independent
+    numpy chain (np.argmax returns the first maximum)."""
+    from tie_streams import planted_prompt
+    d, Bp, Bc = 16, 3, 5
+    rng = np.random.default_rng(60 + Br)
+    K, V, s, n_ev, want = planted_prompt(rng, d, Bp, Bc, Br, n_more=30)
+    u = oracle.Unit(d, 1, Bp, Bc, Br)
+    res = u.prefill_compress(K, V, scores=s)
+    assert np.flatnonzero(res.evicted).tolist() == list(range(n_ev))
+    assert res.targets[:Br].tolist() == [-2] * Br
+    assert res.targets[Br:Br + len(want)].tolist() == want
+    assert res.report.min_merge_gap == 0.0
+    _, _, _, targets = _merge_chain_numpy(K, V, list(range(n_ev)), Br)
+    assert res.targets.tolist() == targets
