@@ -37,6 +37,12 @@
  *     attention weights are averaged for the score [App. C.4].
  *   - Merged (residual) slots are held in fp32 whatever the storage dtype, so
  *     thousands of incremental means do not stall at half precision.
+ *   - Contribution scores [Eq. (score)] are fp32 and ordered as floats of either sign
+ *     (the method itself only produces non-negative ones; -0.0 equals +0.0); equal
+ *     scores are ordered by position.  NaN is not a score: zsm_cache_import_unit
+ *     refuses it (ZSM_ERR_INVALID_ARG) and the prompt pass reports it through the
+ *     sticky status word (ZSM_ERR_DEVICE_CHECK).
+ *   - A handle is not thread-safe: calls on one handle come from one thread at a time.
  */
 #ifndef ZSM_H
 #define ZSM_H
@@ -56,7 +62,8 @@ typedef enum {
     ZSM_ERR_CUDA = 4,             /* a CUDA runtime call failed */
     ZSM_ERR_UNSUPPORTED = 5,      /* shape outside what the kernels are built for */
     ZSM_ERR_DEVICE_CHECK = 6,     /* a device-side consistency check failed */
-    ZSM_ERR_TIMEOUT = 7           /* a bounded device-side wait gave up */
+    ZSM_ERR_TIMEOUT = 7,          /* a bounded device-side wait gave up */
+    ZSM_ERR_NO_MEMORY = 8         /* host memory for the handle could not be allocated */
 } zsm_status_t;
 
 typedef enum { ZSM_F32 = 0, ZSM_F16 = 1, ZSM_BF16 = 2 } zsm_dtype_t;
@@ -111,9 +118,10 @@ zsm_status_t zsm_cache_bytes(const zsm_config_t *cfg, size_t *bytes);
 
 /* Lay the cache out in dev_buf (256-byte aligned, >= zsm_cache_bytes) and
  * return a handle.  Writes the layout tables and empties every unit; blocks
- * until that is done.  The handle keeps dev_buf but never frees it.
+ * until that is done.  The handle keeps dev_buf but never frees it.  Also does
+ * the per-device set-up of zsm_prefill_compress_static (see there).
  * UNSUPPORTED: head_dim, group size or a budget the kernels cannot hold in
- * shared memory. */
+ * shared memory.  NO_MEMORY: the host handle could not be allocated. */
 zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t bytes,
                               zsm_cache_t **out);
 
@@ -155,14 +163,17 @@ zsm_status_t zsm_prefill_compress(zsm_cache_t *c, int32_t layer, const void *K, 
  * cudaMalloc made now would fail, or a latency-critical loop that cannot afford the device
  * synchronisation an allocation may imply.  Arguments, results and status codes are those of
  * zsm_prefill_compress without `workspace`: the scratch is a fixed array of
- * ZSM_STATIC_SCRATCH_BYTES that is part of the library image -- every GPU that loads the
- * library holds those bytes until the process exits -- and the call makes no cudaMalloc,
- * cudaFree or other allocating call.
+ * ZSM_STATIC_SCRATCH_BYTES that is part of the library image -- every GPU on which a cache
+ * has been created holds those bytes until the process exits -- and the call makes no
+ * cudaMalloc, cudaFree or other allocating call.
  *   - ZSM_ERR_BUFFER_TOO_SMALL when the prompt needs more scratch than that
  *     (zsm_prefill_workspace_bytes(c, T, W) tells how much; roughly
  *     batch*n_kv_heads*T*(13 + 4*G*W) bytes).  Nothing is launched then.
- *   - The first call on each device looks up the array's device address (with the cache's
- *     device current, as for every call); make that first call outside any stream capture.
+ *   - Set-up: the array's device address is looked up once per device, and that first look-up
+ *     is also when the device loads the part of the library that holds the array, i.e. when
+ *     the bytes are reserved.  zsm_cache_create does it (a handle is needed for this call
+ *     anyway, so the set-up has always happened on the handle's device); from then on this
+ *     call neither allocates nor synchronises.  Create the cache outside any stream capture.
  *   - All calls on a device share the one array, which keeps what the last call left in
  *     it.  The pass overwrites every entry before it reads it, so nothing needs clearing;
  *     but two calls whose kernels overlap on the GPU (different streams) race on it.
@@ -261,7 +272,8 @@ zsm_status_t zsm_cache_export_unit(zsm_cache_t *c, int32_t layer, int32_t b, int
                                    zsm_stream_t stream);
 
 /* Inverse of export (resume / checkpoint restore): all arrays required, K and V
- * are rounded to the storage dtype.  INVALID_ARG if counters exceed capacity. */
+ * are rounded to the storage dtype.  INVALID_ARG if counters exceed capacity or a
+ * live slot's score is NaN. */
 zsm_status_t zsm_cache_import_unit(zsm_cache_t *c, int32_t layer, int32_t b, int32_t h,
                                    const float *K, const float *V, const float *score,
                                    const int32_t *pos, const float *Kr, const float *Vr,
@@ -272,6 +284,13 @@ zsm_status_t zsm_cache_import_unit(zsm_cache_t *c, int32_t layer, int32_t b, int
  * device-side check or wait has failed since creation or the last call) and
  * clears it. */
 zsm_status_t zsm_last_device_status(zsm_cache_t *c, zsm_stream_t stream);
+
+/* Exercises the device-side failure detector without a fault: launches one CTA whose single
+ * thread waits, with the same bounded wait every kernel of the library uses, on a barrier that
+ * nothing ever arrives at.  After limit_us microseconds (1..1 000 000) the wait gives up, the
+ * kernel records ZSM_ERR_TIMEOUT in the cache's sticky status word and returns normally; the
+ * context stays usable.  Asynchronous; read the outcome with zsm_last_device_status. */
+zsm_status_t zsm_selftest_wait_timeout(zsm_cache_t *c, uint32_t limit_us, zsm_stream_t stream);
 
 /* Launch shape of the fused decode kernel for this layer argument (diagnostics). */
 zsm_status_t zsm_decode_launch_info(const zsm_cache_t *c, int32_t layer, int32_t *grid,

@@ -3,6 +3,12 @@
 Argument marshalling only -- every step of the path runs in the library's CUDA
 kernels.  There is no fallback: if the shared library is missing the import of
 this module raises.  torch is used for device memory and streams.
+
+The C library takes raw pointers and cannot know how large a tensor behind one is,
+so this layer checks every tensor (device, contiguity, dtype, element count)
+against the cache's configuration before it hands the pointer over, and raises
+TypeError / ValueError instead of letting a wrong tensor become an out-of-bounds
+access on the device.
 """
 from __future__ import annotations
 
@@ -23,6 +29,7 @@ ZSM_ERR_CUDA = 4
 ZSM_ERR_UNSUPPORTED = 5
 ZSM_ERR_DEVICE_CHECK = 6
 ZSM_ERR_TIMEOUT = 7
+ZSM_ERR_NO_MEMORY = 8
 ZSM_F32, ZSM_F16, ZSM_BF16 = 0, 1, 2
 DTYPE_CODE = {"f32": ZSM_F32, "f16": ZSM_F16, "bf16": ZSM_BF16,
               torch.float32: ZSM_F32, torch.float16: ZSM_F16, torch.bfloat16: ZSM_BF16}
@@ -35,7 +42,8 @@ SYMBOLS = ["zsm_split_budget", "zsm_cache_bytes", "zsm_cache_create", "zsm_cache
            "zsm_fullkv_status",
            "zsm_decode_step", "zsm_decode_staging_bytes", "zsm_decode_step_host",
            "zsm_unit_capacity", "zsm_cache_export_unit", "zsm_cache_import_unit",
-           "zsm_last_device_status", "zsm_decode_launch_info", "zsm_status_string"]
+           "zsm_last_device_status", "zsm_decode_launch_info", "zsm_status_string",
+           "zsm_selftest_wait_timeout"]
 
 
 class ZsmConfig(C.Structure):
@@ -85,6 +93,7 @@ _lib.zsm_unit_capacity.argtypes = [_vp, _i32, _i32, _pi32, _pi32]
 _lib.zsm_cache_export_unit.argtypes = [_vp, _i32, _i32, _i32] + [_vp] * 8 + [_vp]
 _lib.zsm_cache_import_unit.argtypes = [_vp, _i32, _i32, _i32] + [_vp] * 8 + [_vp]
 _lib.zsm_last_device_status.argtypes = [_vp, _vp]
+_lib.zsm_selftest_wait_timeout.argtypes = [_vp, C.c_uint32, _vp]
 _lib.zsm_decode_launch_info.argtypes = [_vp, _i32, _pi32, _pi32, _pi32]
 for _name in SYMBOLS:
     if _name != "zsm_status_string":
@@ -102,21 +111,73 @@ def _stream(stream=None):
     return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
 
 
-def _dev(t):
+_TORCH_OF_CODE = {ZSM_F32: torch.float32, ZSM_F16: torch.float16, ZSM_BF16: torch.bfloat16}
+
+
+class Cache:
+    """What zsm_cache_create returns: the C handle (passed on wherever a `cache` argument is
+    expected), the shape the checks below need, and a reference to the device buffer so that
+    it outlives the handle."""
+
+    def __init__(self, handle, cfg: ZsmConfig, dev_buf: torch.Tensor):
+        self._as_parameter_ = handle
+        self.buf = dev_buf
+        self.device = dev_buf.device
+        self.n_layers, self.batch = cfg.n_layers, cfg.batch
+        self.n_q_heads, self.n_kv_heads, self.head_dim = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+        self.group = cfg.n_q_heads // cfg.n_kv_heads
+        self.torch_dtype = _TORCH_OF_CODE[cfg.dtype]
+        self._cfg = cfg  # keeps the budget arrays alive
+
+    def units(self, layer: int) -> int:
+        per_layer = self.batch * self.n_kv_heads
+        return per_layer * self.n_layers if layer < 0 else per_layer
+
+
+def _layer_arg(cache: "Cache", layer, allow_all: bool) -> int:
+    layer = int(layer)
+    if layer < (-1 if allow_all else 0) or layer >= cache.n_layers:
+        raise ZsmError(ZSM_ERR_INVALID_ARG, f"layer {layer} of {cache.n_layers}")
+    return layer
+
+
+def _dev(t, name="tensor", dtype=None, numel=None, device=None):
+    """Pointer of a device tensor after checking it is what the call will read or write."""
     if t is None:
         return None
-    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name}: a CUDA tensor is required")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: tensor must be contiguous")
+    if device is not None and t.device != device:
+        raise ValueError(f"{name}: on {t.device}, the cache is on {device}")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name}: dtype {t.dtype}, expected {dtype}")
+    if numel is not None and t.numel() < numel:
+        raise ValueError(f"{name}: {t.numel()} elements, the call needs {numel}")
     return C.c_void_p(t.data_ptr())
 
 
-def _host(a):
+def _host(a, name="array", dtype=None, numel=None):
     if a is None:
         return None
     if isinstance(a, torch.Tensor):
-        assert not a.is_cuda and a.is_contiguous()
+        if a.is_cuda or not a.is_contiguous():
+            raise ValueError(f"{name}: a contiguous host tensor is required")
+        if dtype is not None and a.dtype != dtype:
+            raise TypeError(f"{name}: dtype {a.dtype}, expected {dtype}")
+        if numel is not None and a.numel() < numel:
+            raise ValueError(f"{name}: {a.numel()} elements, the call needs {numel}")
         return C.c_void_p(a.data_ptr())
-    assert a.flags["C_CONTIGUOUS"]
+    if not a.flags["C_CONTIGUOUS"]:
+        raise ValueError(f"{name}: array must be C-contiguous")
+    if numel is not None and a.size < numel:
+        raise ValueError(f"{name}: {a.size} elements, the call needs {numel}")
     return C.c_void_p(a.ctypes.data)
+
+
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
 
 
 def zsm_status_string(status: int) -> str:
@@ -151,11 +212,11 @@ def zsm_cache_bytes(cfg: ZsmConfig) -> int:
     return n.value
 
 
-def zsm_cache_create(cfg: ZsmConfig, dev_buf: torch.Tensor):
+def zsm_cache_create(cfg: ZsmConfig, dev_buf: torch.Tensor) -> Cache:
     h = _vp()
-    _check(_lib.zsm_cache_create(C.byref(cfg), _dev(dev_buf), dev_buf.numel() * dev_buf.element_size(),
-                                 C.byref(h)), "zsm_cache_create")
-    return h
+    _check(_lib.zsm_cache_create(C.byref(cfg), _dev(dev_buf, "dev_buf"), _nbytes(dev_buf), C.byref(h)),
+           "zsm_cache_create")
+    return Cache(h, cfg, dev_buf)
 
 
 def zsm_cache_reset(cache, stream=None):
@@ -164,6 +225,8 @@ def zsm_cache_reset(cache, stream=None):
 
 def zsm_cache_free(cache):
     _check(_lib.zsm_cache_free(cache), "zsm_cache_free")
+    if isinstance(cache, Cache):
+        cache._as_parameter_ = None   # a freed handle must never reach the library again
 
 
 def zsm_prefill_workspace_bytes(cache, T: int, W: int) -> int:
@@ -173,13 +236,28 @@ def zsm_prefill_workspace_bytes(cache, T: int, W: int) -> int:
     return n.value
 
 
+def _prefill_args(cache: Cache, layer, K, V, Qw, scores, T, W, dbg_scores, dbg_evicted, dbg_targets):
+    layer, T, W = _layer_arg(cache, layer, False), int(T), int(W)
+    if T < 1 or (Qw is not None and not 1 <= W <= T):
+        raise ZsmError(ZSM_ERR_INVALID_ARG, f"T = {T}, W = {W}")
+    dt, dev, d = cache.torch_dtype, cache.device, cache.head_dim
+    rows = cache.batch * cache.n_kv_heads * T
+    return (layer, _dev(K, "K", dt, rows * d, dev), _dev(V, "V", dt, rows * d, dev),
+            _dev(Qw, "Qw", dt, cache.batch * cache.n_q_heads * W * d, dev),
+            _dev(scores, "scores", torch.float32, rows, dev), T, W,
+            _dev(dbg_scores, "dbg_scores", torch.float32, rows, dev),
+            _dev(dbg_evicted, "dbg_evicted", torch.uint8, rows, dev),
+            _dev(dbg_targets, "dbg_targets", torch.int32, rows, dev))
+
+
 def zsm_prefill_compress(cache, layer, K, V, Qw, scores, T, W, workspace, dbg_scores=None,
                          dbg_evicted=None, dbg_targets=None, stream=None):
-    _check(_lib.zsm_prefill_compress(cache, int(layer), _dev(K), _dev(V), _dev(Qw), _dev(scores),
-                                     int(T), int(W), _dev(workspace),
-                                     workspace.numel() * workspace.element_size(),
-                                     _dev(dbg_scores), _dev(dbg_evicted), _dev(dbg_targets),
-                                     _stream(stream)), "zsm_prefill_compress")
+    layer, pK, pV, pQ, pS, T, W, d1, d2, d3 = _prefill_args(cache, layer, K, V, Qw, scores, T, W,
+                                                           dbg_scores, dbg_evicted, dbg_targets)
+    _check(_lib.zsm_prefill_compress(cache, layer, pK, pV, pQ, pS, T, W,
+                                     _dev(workspace, "workspace", device=cache.device),
+                                     _nbytes(workspace), d1, d2, d3, _stream(stream)),
+           "zsm_prefill_compress")
 
 
 ZSM_STATIC_SCRATCH_BYTES = 16 << 20
@@ -191,9 +269,12 @@ def zsm_prefill_compress_static(cache, layer, K, V, Qw, scores, T, W, dbg_scores
     tensor, for callers that cannot allocate device memory at the time of the call.  Raises
     ZsmError(ZSM_ERR_BUFFER_TOO_SMALL) when the prompt needs more than
     ZSM_STATIC_SCRATCH_BYTES; calls on different streams must not overlap."""
-    _check(_lib.zsm_prefill_compress_static(cache, int(layer), _dev(K), _dev(V), _dev(Qw),
-                                            _dev(scores), int(T), int(W), _dev(dbg_scores),
-                                            _dev(dbg_evicted), _dev(dbg_targets),
+    need = zsm_prefill_workspace_bytes(cache, T, W if Qw is not None else 0)
+    if need > ZSM_STATIC_SCRATCH_BYTES:   # before any tensor is looked at, as in the library
+        raise ZsmError(ZSM_ERR_BUFFER_TOO_SMALL, "zsm_prefill_compress_static")
+    layer, pK, pV, pQ, pS, T, W, d1, d2, d3 = _prefill_args(cache, layer, K, V, Qw, scores, T, W,
+                                                           dbg_scores, dbg_evicted, dbg_targets)
+    _check(_lib.zsm_prefill_compress_static(cache, layer, pK, pV, pQ, pS, T, W, d1, d2, d3,
                                             _stream(stream)), "zsm_prefill_compress_static")
 
 
@@ -207,17 +288,36 @@ def zsm_prefill_scores_full_workspace_bytes(cache, T: int) -> int:
 def zsm_prefill_scores_full(cache, K, Q, T, scores, workspace=None, lse=None, stream=None):
     """Full-history prompt scores (every prompt query scores every earlier key) into `scores`
     fp32 [batch][n_kv_heads][T]; `lse` optionally supplies the rows' log-sum-exp."""
-    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    _check(_lib.zsm_prefill_scores_full(cache, _dev(K), _dev(Q), _dev(lse), int(T), _dev(scores),
-                                        _dev(workspace), nbytes, _stream(stream)),
-           "zsm_prefill_scores_full")
+    T = int(T)
+    dt, dev, d = cache.torch_dtype, cache.device, cache.head_dim
+    _check(_lib.zsm_prefill_scores_full(
+        cache, _dev(K, "K", dt, cache.batch * cache.n_kv_heads * T * d, dev),
+        _dev(Q, "Q", dt, cache.batch * cache.n_q_heads * T * d, dev),
+        _dev(lse, "lse", torch.float32, cache.batch * cache.n_q_heads * T, dev), T,
+        _dev(scores, "scores", torch.float32, cache.batch * cache.n_kv_heads * T, dev),
+        _dev(workspace, "workspace", device=dev), _nbytes(workspace), _stream(stream)),
+        "zsm_prefill_scores_full")
+
+
+def _decode_args(cache: Cache, layer, q, k_new, v_new, out, host: bool):
+    layer = _layer_arg(cache, layer, True)
+    nu, d, dt = cache.units(layer), cache.head_dim, cache.torch_dtype
+    if host:
+        return (layer, _host(q, "q", dt, nu * cache.group * d), _host(k_new, "k_new", dt, nu * d),
+                _host(v_new, "v_new", dt, nu * d), _host(out, "out", dt, nu * cache.group * d))
+    dev = cache.device
+    return (layer, _dev(q, "q", dt, nu * cache.group * d, dev), _dev(k_new, "k_new", dt, nu * d, dev),
+            _dev(v_new, "v_new", dt, nu * d, dev), _dev(out, "out", dt, nu * cache.group * d, dev))
 
 
 def zsm_decode_step(cache, layer, q, k_new, v_new, out, victim_pos=None, merge_slot=None,
                     stream=None):
-    _check(_lib.zsm_decode_step(cache, int(layer), _dev(q), _dev(k_new), _dev(v_new), _dev(out),
-                                _dev(victim_pos), _dev(merge_slot), _stream(stream)),
-           "zsm_decode_step")
+    layer, pq, pk, pv, po = _decode_args(cache, layer, q, k_new, v_new, out, host=False)
+    nu = cache.units(layer)
+    _check(_lib.zsm_decode_step(cache, layer, pq, pk, pv, po,
+                                _dev(victim_pos, "victim_pos", torch.int32, nu, cache.device),
+                                _dev(merge_slot, "merge_slot", torch.int32, nu, cache.device),
+                                _stream(stream)), "zsm_decode_step")
 
 
 def zsm_fullkv_workspace_bytes(n_units: int, group: int, head_dim: int, T: int) -> int:
@@ -232,14 +332,19 @@ def zsm_fullkv_decode(K, V, q, out, workspace, softmax_scale=0.0, stream=None):
     [units, G, d] device tensors of one 16-bit dtype."""
     n_units, T, d = K.shape
     G = q.shape[1]
-    _check(_lib.zsm_fullkv_decode(int(DTYPE_CODE[K.dtype]), int(n_units), int(G), int(d), int(T),
-                                  _dev(K), _dev(V), _dev(q), _dev(out), float(softmax_scale),
-                                  _dev(workspace), workspace.numel() * workspace.element_size(),
+    if tuple(V.shape) != (n_units, T, d) or tuple(q.shape) != (n_units, G, d) or \
+            tuple(out.shape) != (n_units, G, d):
+        raise ValueError("zsm_fullkv_decode: K, V [units, T, d] and q, out [units, G, d] disagree")
+    dt, dev = K.dtype, K.device
+    _check(_lib.zsm_fullkv_decode(int(DTYPE_CODE[dt]), int(n_units), int(G), int(d), int(T),
+                                  _dev(K, "K"), _dev(V, "V", dt, device=dev), _dev(q, "q", dt, device=dev),
+                                  _dev(out, "out", dt, device=dev), float(softmax_scale),
+                                  _dev(workspace, "workspace", device=dev), _nbytes(workspace),
                                   _stream(stream)), "zsm_fullkv_decode")
 
 
 def zsm_fullkv_status(workspace, stream=None) -> int:
-    return int(_lib.zsm_fullkv_status(_dev(workspace), _stream(stream)))
+    return int(_lib.zsm_fullkv_status(_dev(workspace, "workspace"), _stream(stream)))
 
 
 def zsm_decode_staging_bytes(cache, layer) -> int:
@@ -250,10 +355,11 @@ def zsm_decode_staging_bytes(cache, layer) -> int:
 
 def zsm_decode_step_host(cache, layer, q_host, k_new_host, v_new_host, out_host, staging,
                          stream=None):
-    _check(_lib.zsm_decode_step_host(cache, int(layer), _host(q_host), _host(k_new_host),
-                                     _host(v_new_host), _host(out_host), _dev(staging),
-                                     staging.numel() * staging.element_size(), _stream(stream)),
-           "zsm_decode_step_host")
+    layer, pq, pk, pv, po = _decode_args(cache, layer, q_host, k_new_host, v_new_host, out_host,
+                                         host=True)
+    _check(_lib.zsm_decode_step_host(cache, layer, pq, pk, pv, po,
+                                     _dev(staging, "staging", device=cache.device), _nbytes(staging),
+                                     _stream(stream)), "zsm_decode_step_host")
 
 
 def zsm_unit_capacity(cache, layer, h):
@@ -307,6 +413,12 @@ def zsm_cache_import_unit(cache, layer, b, h, head_dim, state, stream=None):
 
 def zsm_last_device_status(cache, stream=None) -> int:
     return int(_lib.zsm_last_device_status(cache, _stream(stream)))
+
+
+def zsm_selftest_wait_timeout(cache, limit_us: int, stream=None):
+    """Launches the library's wait self-test: one bounded wait that can only end by its limit."""
+    _check(_lib.zsm_selftest_wait_timeout(cache, int(limit_us), _stream(stream)),
+           "zsm_selftest_wait_timeout")
 
 
 def zsm_decode_launch_info(cache, layer):

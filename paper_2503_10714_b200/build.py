@@ -11,7 +11,7 @@ LIB = os.path.join(HERE, "libzsm.so")
 SOURCES = ["zsm_api.cu", "zsm_decode.cu", "zsm_decode_split.cu", "zsm_prefill.cu",
            "zsm_prefill_full.cu", "zsm_noalloc.cu", "zsm_fullkv.cu"]
 HEADERS = ["zsm_common.cuh", "zsm_decode.cuh", "zsm_decode_split.cuh", "zsm_prefill.cuh",
-           "zsm_prefill_full.cuh"]
+           "zsm_prefill_full.cuh", "zsm_noalloc.cuh"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "-shared"]
 

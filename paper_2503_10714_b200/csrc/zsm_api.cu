@@ -11,6 +11,7 @@
 
 #include "zsm_decode.cuh"
 #include "zsm_decode_split.cuh"
+#include "zsm_noalloc.cuh"
 #include "zsm_prefill.cuh"
 #include "zsm_prefill_full.cuh"
 
@@ -238,6 +239,7 @@ const char *zsm_status_string(zsm_status_t s) {
         case ZSM_ERR_UNSUPPORTED: return "unsupported shape";
         case ZSM_ERR_DEVICE_CHECK: return "device-side check failed";
         case ZSM_ERR_TIMEOUT: return "device-side wait timed out";
+        case ZSM_ERR_NO_MEMORY: return "out of host memory";
     }
     return "unknown status";
 }
@@ -293,7 +295,7 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
     if (bytes < need) return ZSM_ERR_BUFFER_TOO_SMALL;
 
     zsm_cache *c = new (std::nothrow) zsm_cache();
-    if (!c) return ZSM_ERR_CUDA;
+    if (!c) return ZSM_ERR_NO_MEMORY;
     c->s = make_shape(cfg);
     const Shape &s = c->s;
     c->lambda = cfg->lambda;
@@ -455,6 +457,11 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
         delete c;
         return ZSM_ERR_CUDA;
     }
+    // Set-up of zsm_prefill_compress_static for this device, here because this call blocks and
+    // may allocate anyway.  A failure is not this call's: the static entry point retries and
+    // reports it.
+    (void)static_scratch_setup();
+    (void)cudaGetLastError();
     *out = c;
     return ZSM_OK;
 }
@@ -740,6 +747,8 @@ zsm_status_t zsm_cache_import_unit(zsm_cache_t *c, int32_t layer, int32_t b, int
     if (counters[0] < 0 || (size_t)counters[0] > cap || counters[1] < 0 || counters[1] > d.Br ||
         counters[2] < counters[0])
         return ZSM_ERR_INVALID_ARG;
+    for (int32_t i = 0; i < counters[0]; ++i)
+        if (std::isnan(score[i])) return ZSM_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaStreamSynchronize(cs) != cudaSuccess) return ZSM_ERR_CUDA;
     std::vector<uint8_t> raw(cap * s.row_bytes);
@@ -775,6 +784,13 @@ zsm_status_t zsm_cache_import_unit(zsm_cache_t *c, int32_t layer, int32_t b, int
                        sizeof(uc), cudaMemcpyHostToDevice);
     }
     return cuda_status(e);
+}
+
+zsm_status_t zsm_selftest_wait_timeout(zsm_cache_t *c, uint32_t limit_us, zsm_stream_t stream) {
+    if (!c || limit_us < 1u || limit_us > 1000000u) return ZSM_ERR_INVALID_ARG;
+    const int rc = launch_wait_selftest(reinterpret_cast<int32_t *>(c->base + c->lay.status),
+                                        limit_us, static_cast<cudaStream_t>(stream));
+    return rc == 0 ? ZSM_OK : ZSM_ERR_CUDA;
 }
 
 zsm_status_t zsm_last_device_status(zsm_cache_t *c, zsm_stream_t stream) {

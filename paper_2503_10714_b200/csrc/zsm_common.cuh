@@ -59,6 +59,14 @@ __device__ __forceinline__ void dev_set_status(int32_t *status, int32_t code, in
     }
 }
 
+// Monotone map fp32 -> uint32: a < b as floats  <=>  score_order_bits(a) < score_order_bits(b)
+// as unsigned integers, for every sign (-0.0 is taken as +0.0 first, so the two zeros tie as
+// they do in a float comparison).  The victim search orders 64-bit keys (these bits, position).
+__device__ __forceinline__ uint32_t score_order_bits(float s) {
+    const uint32_t u = __float_as_uint(s + 0.0f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
 // ---------------------------------------------------------------------------
 // Storage-type helpers: 16 bytes = EPL elements, widened to fp32.
 // ---------------------------------------------------------------------------
@@ -186,7 +194,7 @@ constexpr uint32_t kSuspendHintNs = 20000u;        // per poll
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity,
                                                   volatile int32_t *abort_flag, int32_t *status,
-                                                  int32_t where) {
+                                                  int32_t where, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     uint32_t polls = 0;
@@ -195,7 +203,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
         ++polls;
         if ((polls & 7u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 dev_set_status(status, DEV_ERR_TIMEOUT, where, static_cast<int32_t>(blockIdx.x));
                 *abort_flag = 1;
                 __threadfence_block();

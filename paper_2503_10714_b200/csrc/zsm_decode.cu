@@ -776,7 +776,7 @@ __global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 
                 const int32_t pj = tp[k];
                 if (evict && pj <= cut) {
                     const uint64_t key =
-                        (static_cast<uint64_t>(__float_as_uint(s_new)) << 32) | (uint32_t)pj;
+                        (static_cast<uint64_t>(score_order_bits(s_new)) << 32) | (uint32_t)pj;
                     if (key < best) {
                         best = key;
                         best_slot = j0 + k;
@@ -793,7 +793,7 @@ __global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 
         if (evict) {
             if (tid == 0 && d.Bp == 0) {
                 const uint64_t key =
-                    (static_cast<uint64_t>(__float_as_uint(s_tok)) << 32) | (uint32_t)Tpos;
+                    (static_cast<uint64_t>(score_order_bits(s_tok)) << 32) | (uint32_t)Tpos;
                 if (key < best) {
                     best = key;
                     best_slot = -2;
@@ -1041,6 +1041,28 @@ int prepare_decode_fused(int dtype, int D, int G, int smem_bytes, int threads,
                          int *max_ctas_per_sm) {
     ZSM_DISPATCH(prepare_one, smem_bytes, threads, max_ctas_per_sm);
     return -1;
+}
+
+namespace {
+constexpr int32_t W_SELFTEST = 99;
+
+// The failure detector's own test: the wait below can only end by its time limit.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(int32_t *status, uint32_t limit_us) {
+    __shared__ uint64_t bar;
+    __shared__ int32_t abort_flag;
+    if (threadIdx.x != 0) return;
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // phase 0 of a barrier with one expected arrival never completes here
+    (void)mbar_wait_bounded(&bar, 0u, &abort_flag, status, W_SELFTEST,
+                            static_cast<uint64_t>(limit_us) * 1000ull);
+}
+}  // namespace
+
+int launch_wait_selftest(int32_t *status, uint32_t limit_us, cudaStream_t stream) {
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_us);
+    return static_cast<int>(cudaGetLastError());
 }
 
 }  // namespace zsm

@@ -76,4 +76,8 @@ int launch_decode_fused(int dtype, int D, int G, const DecodeParams &p, int grid
 int prepare_decode_fused(int dtype, int D, int G, int smem_bytes, int threads,
                          int *max_ctas_per_sm);
 
+// One CTA, one thread, waiting with the library's bounded wait on a barrier nothing arrives at;
+// gives up after limit_us and records DEV_ERR_TIMEOUT in *status.  Returns a cudaError_t as int.
+int launch_wait_selftest(int32_t *status, uint32_t limit_us, cudaStream_t stream);
+
 }  // namespace zsm

@@ -732,7 +732,7 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
             score_g[j0 + k] = s_new;
             const int32_t pj = tp[k];
             if (evict && pj <= cut) {
-                const uint64_t key = (static_cast<uint64_t>(__float_as_uint(s_new)) << 32) | (uint32_t)pj;
+                const uint64_t key = (static_cast<uint64_t>(score_order_bits(s_new)) << 32) | (uint32_t)pj;
                 if (key < best) {
                     best = key;
                     best_slot = row_lo + j0 + k;
@@ -749,7 +749,7 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     }
     if (evict) {
         if (tid == 0 && rank == 0 && d.Bp == 0) {
-            const uint64_t key = (static_cast<uint64_t>(__float_as_uint(s_tok)) << 32) | (uint32_t)Tpos;
+            const uint64_t key = (static_cast<uint64_t>(score_order_bits(s_tok)) << 32) | (uint32_t)Tpos;
             if (key < best) {
                 best = key;
                 best_slot = -2;

@@ -4,6 +4,8 @@
 
 #include <cuda_runtime.h>
 
+#include "zsm_noalloc.cuh"
+
 #include <mutex>
 
 namespace {
@@ -17,7 +19,10 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
 void *g_scratch_addr[kMaxDevices];  // device address of the array on each device, once looked up
 
-// Device address of the array on the current device; looked up once per device.
+// Device address of the array on the current device; looked up once per device.  The first
+// look-up on a device is also the first use of this file's module there: under lazy module
+// loading that is when the device reserves the array's bytes, so it belongs to set-up time
+// (zsm_cache_create calls it through zsm::static_scratch_setup), not to the no-allocation call.
 zsm_status_t static_scratch(void **out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ZSM_ERR_CUDA;
@@ -32,6 +37,13 @@ zsm_status_t static_scratch(void **out) {
 }
 
 }  // namespace
+
+namespace zsm {
+int static_scratch_setup() {
+    void *p = nullptr;
+    return static_scratch(&p) == ZSM_OK ? 0 : 1;
+}
+}  // namespace zsm
 
 extern "C" zsm_status_t zsm_prefill_compress_static(zsm_cache_t *c, int32_t layer, const void *K,
                                                     const void *V, const void *Qw,

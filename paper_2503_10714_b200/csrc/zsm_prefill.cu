@@ -19,12 +19,6 @@ namespace zsm {
 
 namespace {
 
-__device__ __forceinline__ uint32_t order_bits(float s) {
-    // monotone map float -> uint32 (also right for negative inputs)
-    const uint32_t u = __float_as_uint(s);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 // ---------------------------------------------------------------------------
 // P1a: logits of one chunk of prompt positions against every window query.
 // grid (chunks, units), 256 threads: thread (tx, ty) owns positions tx+32i and
@@ -312,7 +306,7 @@ __global__ void __launch_bounds__(1024) prefill_select_kernel(const PrefillParam
     const int tid = threadIdx.x;
 
     auto key_of = [&](int t) -> uint64_t {
-        return (static_cast<uint64_t>(order_bits(s[t])) << 32) | static_cast<uint32_t>(t);
+        return (static_cast<uint64_t>(score_order_bits(s[t])) << 32) | static_cast<uint32_t>(t);
     };
 
     uint64_t thr = 0;
@@ -357,6 +351,7 @@ __global__ void __launch_bounds__(1024) prefill_select_kernel(const PrefillParam
         const int t = t0 + tid;
         const bool in = t < T_len;
         const bool ev = in && n_ev > 0 && t < n_cand && key_of(t) <= thr;
+        if (in && s[t] != s[t]) dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 5);  // NaN score
         const bool kp = in && !ev;
         if (in) flags[t] = ev ? 1 : 0;
         const uint32_t be = __ballot_sync(0xffffffffu, ev);

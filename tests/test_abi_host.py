@@ -75,6 +75,8 @@ def test_invalid_configs_are_rejected_on_the_host(zb):
             zb.zsm_cache_bytes(zb.make_config(**{**ok, **patch}))
         assert e.value.status == zb.ZSM_ERR_INVALID_ARG
     assert zb.zsm_status_string(zb.ZSM_ERR_TIMEOUT) == "device-side wait timed out"
+    assert zb.zsm_status_string(zb.ZSM_ERR_NO_MEMORY) == "out of host memory"
+    assert zb._lib.zsm_selftest_wait_timeout(None, 1000, None) == zb.ZSM_ERR_INVALID_ARG
     # null handles never reach CUDA
     assert zb._lib.zsm_cache_free(None) == zb.ZSM_ERR_INVALID_ARG
     assert zb._lib.zsm_decode_step(None, 0, None, None, None, None, None, None, None) == zb.ZSM_ERR_INVALID_ARG

@@ -202,8 +202,10 @@ def test_argument_errors_reach_the_caller(zb):
         with pytest.raises(zb.ZsmError) as e:
             zb.zsm_decode_step(c.h, 7, q, k, v, c.out_all)
         assert e.value.status == zb.ZSM_ERR_INVALID_ARG
-        with pytest.raises(zb.ZsmError):
-            zb.zsm_decode_step(c.h, -1, q.view(-1)[1:], k, v, c.out_all)   # misaligned pointer
+        big = torch.zeros(q.numel() + 8, dtype=q.dtype, device="cuda")
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_decode_step(c.h, -1, big[1:], k, v, c.out_all)          # misaligned pointer
+        assert e.value.status == zb.ZSM_ERR_INVALID_ARG
         small = torch.empty(16, dtype=torch.uint8, device="cuda")
         with pytest.raises(zb.ZsmError) as e:
             zb.zsm_cache_create(c.cfg, small)
@@ -215,6 +217,118 @@ def test_argument_errors_reach_the_caller(zb):
         assert e.value.status == zb.ZSM_ERR_UNSUPPORTED
     finally:
         c.close()
+
+
+def test_wrong_tensors_are_refused_before_they_reach_the_device(zb):
+    """The binding checks every tensor against the cache's shape: a short, wrongly typed, host
+    or non-contiguous tensor raises instead of becoming an out-of-bounds access in a kernel."""
+    w = SMALL.replace(dtype="f16", head_dim=128)
+    c = GpuCache(zb, w, np.full((2, 2), 4), np.full((2, 2), 4), np.full((2, 2), 1))
+    try:
+        q, k, v = (t.cuda() for t in wl.decode_inputs(w, 0))
+        out = c.out_all
+        with pytest.raises(ValueError):
+            zb.zsm_decode_step(c.h, -1, q[0], k, v, out)                   # one layer's q for all layers
+        with pytest.raises(ValueError):
+            zb.zsm_decode_step(c.h, -1, q, k[:, :1], v, out)               # short k_new
+        with pytest.raises(TypeError):
+            zb.zsm_decode_step(c.h, -1, q.float(), k, v, out)              # wrong dtype
+        with pytest.raises(TypeError):
+            zb.zsm_decode_step(c.h, -1, q.cpu(), k, v, out)                # host tensor
+        with pytest.raises(ValueError):
+            zb.zsm_decode_step(c.h, -1, q.transpose(1, 2), k, v, out)      # not contiguous
+        with pytest.raises(TypeError):
+            zb.zsm_decode_step(c.h, -1, q, k, v, out, victim_pos=torch.zeros(8, device="cuda"))
+        with pytest.raises(ValueError):
+            zb.zsm_decode_step(c.h, 0, q[0], k[0], v[0], out[0],
+                               merge_slot=torch.zeros(1, dtype=torch.int32, device="cuda"))
+        T, W = 64, 8
+        K = torch.zeros(w.batch, w.n_kv_heads, T, 128, dtype=torch.float16, device="cuda")
+        Qw = torch.zeros(w.batch, w.n_q_heads, W, 128, dtype=torch.float16, device="cuda")
+        ws = torch.empty(zb.zsm_prefill_workspace_bytes(c.h, T, W), dtype=torch.uint8, device="cuda")
+        with pytest.raises(ValueError):
+            zb.zsm_prefill_compress(c.h, 0, K[:, :, :32].contiguous(), K, Qw, None, T, W, ws)
+        with pytest.raises(ValueError):
+            zb.zsm_prefill_compress(c.h, 0, K, K, Qw[:, :1].contiguous(), None, T, W, ws)
+        with pytest.raises(TypeError):
+            zb.zsm_prefill_compress(c.h, 0, K, K, None, torch.zeros(w.batch, w.n_kv_heads, T,
+                                                                    dtype=torch.float16, device="cuda"),
+                                    T, 0, ws)
+        with pytest.raises(ValueError):
+            zb.zsm_prefill_compress(c.h, 0, K, K, Qw, None, T, W, ws,
+                                    dbg_targets=torch.zeros(T, dtype=torch.int32, device="cuda"))
+        zb.zsm_prefill_compress(c.h, 0, K, K, Qw, None, T, W, ws)          # and the right ones pass
+        zb.zsm_decode_step(c.h, -1, q, k, v, out)
+        assert c.status() == 0
+        assert c.h.buf is c.buf                                            # the handle keeps the buffer
+    finally:
+        c.close()
+
+
+def test_bounded_wait_gives_up_and_reports_timeout(zb):
+    """The device-side failure detector, run without a fault: a wait that nothing can satisfy
+    ends by its time limit, the kernel returns, the sticky status says ZSM_ERR_TIMEOUT, and the
+    cache decodes normally afterwards."""
+    w = SMALL.replace(dtype="f16", head_dim=128)
+    c = GpuCache(zb, w, np.full((2, 2), 4), np.full((2, 2), 4), np.full((2, 2), 1))
+    try:
+        assert c.status() == 0
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        zb.zsm_selftest_wait_timeout(c.h, 3000)          # 3 ms
+        t1.record()
+        assert c.status() == zb.ZSM_ERR_TIMEOUT
+        assert 2.5 <= t0.elapsed_time(t1) <= 200.0, "the wait must last about its limit, then end"
+        assert c.status() == 0                            # reading clears it
+        q, k, v = (t.cuda() for t in wl.decode_inputs(w, 0))
+        c.decode(q, k, v)
+        assert c.status() == 0
+        with pytest.raises(zb.ZsmError):
+            zb.zsm_selftest_wait_timeout(c.h, 0)
+    finally:
+        c.close()
+
+
+def test_scores_of_either_sign_order_as_floats(zb, oracle):
+    """Scores handed in from outside (import, caller-supplied prompt scores) may be negative or
+    -0.0: the victim is still the lowest float, not the lowest bit pattern; NaN is refused."""
+    w = wl.Workload("signed", 1, 1, 2, 1, 128, "f16", 0, 0, 0, None, 19)
+    cache = GpuCache(zb, w, [[2]], [[6]], [[2]], lam=1.0)
+    stats = ParityStats()
+    try:
+        rs = np.random.RandomState(7)
+        T = 40
+        K = torch.from_numpy(rs.randn(T, 128)).to(torch.float16)
+        V = torch.from_numpy(rs.randn(T, 128)).to(torch.float16)
+        scores = np.linspace(-30.0, 30.0, T).astype(np.float32)
+        rs.shuffle(scores)
+        scores[5], scores[9] = -0.0, 0.0
+        unit = oracle_unit_for(oracle, cache, 0, 0)
+        unit.prefill_compress(f64(K), f64(V), scores=scores)
+        dbg = cache.prefill(0, K[None, None].cuda(), V[None, None].cuda(), None,
+                            torch.from_numpy(scores)[None, None].cuda())
+        state_check(unit, cache.export(0, 0, 0), stats, tag="signed scores, prompt pass")
+        for step in range(12):
+            q, k, v = wl.decode_inputs(w, step)
+            out, vic, slot = cache.decode(q.cuda(), k.cuda(), v.cuda())
+            oracle_step_check(unit, f64(q)[0, 0], f64(k)[0, 0, 0], f64(v)[0, 0, 0], f64(out)[0, 0],
+                              int(vic.cpu()[0, 0, 0]), int(slot.cpu()[0, 0, 0]), w.dtype, stats,
+                              tag=f"signed scores step {step}")
+        assert stats.selections >= 10 and stats.victim_near_ties == 0
+        assert cache.status() == 0
+        st = cache.export(0, 0, 0)
+        st["score"] = st["score"].copy()
+        st["score"][1] = np.nan
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_cache_import_unit(cache.h, 0, 0, 0, 128, st)
+        assert e.value.status == zb.ZSM_ERR_INVALID_ARG
+        bad = torch.from_numpy(scores.copy())
+        bad[3] = float("nan")
+        cache.prefill(0, K[None, None].cuda(), V[None, None].cuda(), None, bad[None, None].cuda())
+        assert cache.status() == zb.ZSM_ERR_DEVICE_CHECK
+    finally:
+        cache.close()
 
 
 def test_caches_of_one_shape_and_different_budgets_coexist(zb):

@@ -72,7 +72,7 @@ def test_many_equal_scores_across_tiles_and_warps(zb, form, dtype, d, G):
         victims = []
         for i in range(n_same + n_hot):
             _, vic, _ = cache.decode(q, tok(1.0 if i < n_same else 6.0), vv)
-            victims.append(vic)
+            victims.append(vic.clone())
         victims = torch.stack(victims).flatten().cpu().tolist()
         assert victims == [-1] * n_same + list(range(n_hot))
         assert cache.status() == 0

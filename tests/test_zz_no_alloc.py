@@ -69,6 +69,28 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row(zb):
         ref.close(), sta.close()
 
 
+def test_static_scratch_call_leaves_device_memory_alone(zb):
+    """What the entry point is for: once a cache exists on the device (its creation does the
+    one-time look-up of the array, which is when the device reserves the array's bytes), a call
+    changes neither the free device memory nor what torch's allocator holds."""
+    w = wl.Workload("noalloc_mem", 1, 2, 4, 2, 128, "f16", 500, 0, 16, None, 33)
+    c = GpuCache(zb, w, np.full((1, 2), 16), np.full((1, 2), 20), np.full((1, 2), 3))
+    try:
+        K, V, Qw = (t.cuda() for t in wl.prompt(w, 0))
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        reserved0 = torch.cuda.memory_reserved()
+        for _ in range(3):
+            zb.zsm_prefill_compress_static(c.h, 0, K, V, Qw, None, w.prompt_len, w.window)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0, f"free device memory changed by {free0 - free1} bytes"
+        assert torch.cuda.memory_reserved() == reserved0
+        assert c.status() == 0
+    finally:
+        c.close()
+
+
 def test_prompt_beyond_the_fixed_scratch_is_refused(zb):
     w = wl.Workload("noalloc_big", 1, 4, 8, 8, 128, "f16", 0, 0, 0, None, 32)
     c = GpuCache(zb, w, np.full((1, 8), 8), np.full((1, 8), 8), np.full((1, 8), 1))
