@@ -8,6 +8,9 @@ compared element by element; the remaining units are covered by properties that 
 any size (occupancy, position bookkeeping, device status).  Inputs are drawn on the GPU by
 the shared seeded recipe; the sampled units' inputs are copied to the host for the oracle.
 """
+import json
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -25,6 +28,9 @@ def zb():
         pytest.skip("no CUDA device")
     from paper_2503_10714_b200 import binding
     return binding
+
+
+NEAR_TIE_BOUND = 1e-3   # near ties per decision (eviction or merge target) the tests accept
 
 
 def run_full_size(zb, oracle, w, n_sample, steps, seed=0, layer_mode=-1):
@@ -108,7 +114,23 @@ def run_full_size(zb, oracle, w, n_sample, steps, seed=0, layer_mode=-1):
     finally:
         cache.close()
     assert stats.exact_tie_breaches == 0
-    print(w.name, stats)
+    # Near ties (the two sides' fp32 values within 1e-4 relative of each other, the oracle then
+    # follows the kernel) are what different summation orders must produce now and then -- a few
+    # per ten thousand decisions at most.  More would mean the kernel's arithmetic drifts.
+    decisions = stats.selections + stats.merges
+    near = stats.victim_near_ties + stats.merge_near_ties
+    assert near <= max(2, NEAR_TIE_BOUND * decisions), \
+        f"{w.name}: {near} near ties in {decisions} decisions"
+    record = dict(workload=w.name, launches="per layer" if layer_mode == "each" else "all layers",
+                  sampled_units=len(sample), steps=steps, selections=int(stats.selections),
+                  merges=int(stats.merges), victim_near_ties=int(stats.victim_near_ties),
+                  merge_near_ties=int(stats.merge_near_ties), exact_tie_breaches=0,
+                  max_out_err=stats.max_out_err, max_score_rel=stats.max_score_rel,
+                  max_res_err=stats.max_res_err)
+    print("parity counts:", json.dumps(record))
+    if os.environ.get("ZSM_PARITY_COUNTS_FILE"):
+        with open(os.environ["ZSM_PARITY_COUNTS_FILE"], "a") as f:
+            f.write(json.dumps(record) + "\n")
     return stats
 
 

@@ -93,6 +93,32 @@ def test_full_scores_against_the_definition(zb, T, lam):
         cache.close()
 
 
+@pytest.mark.parametrize("dtype,head_dim,group,T", [("bf16", 128, 4, 8192 + 77), ("f16", 64, 2, 8192 + 130)])
+def test_full_scores_at_long_prompts(zb, oracle, dtype, head_dim, group, T):
+    """A prompt of more than 64 key blocks with grouped heads: every CTA walks hundreds of
+    (tile, head) items, so the tile ring, the exponent-offset ring and the accumulator phases
+    wrap many times.  The oracle's full-history pass is quadratic, so one sampled head per
+    sequence is recomputed; the rest are held to what holds for any input (finite, positive,
+    and the column sums of a softmax matrix add up to the sum of the decay weights)."""
+    w = wl.Workload("fulllong", 1, 2, 3 * group, 3, head_dim, dtype, T, 0, T, None, 38)
+    cache = GpuCache(zb, w, [[8] * 3], [[20] * 3], [[2] * 3])
+    try:
+        K, V, Q = wl.prompt(w, 0)
+        s_gpu, _ = full_scores(zb, cache, K.cuda(), Q.cuda())
+        assert cache.status() == 0
+        s_gpu = s_gpu.cpu().numpy().astype(np.float64)
+        assert np.isfinite(s_gpu).all() and (s_gpu > 0).all()
+        lam = float(np.float32(cache.lam))
+        total = sum(lam ** (T - 1 - q) for q in range(T))        # each softmax row sums to one
+        np.testing.assert_allclose(s_gpu.sum(axis=-1), total, rtol=1e-5)
+        for b, h in [(0, 1), (1, 2)]:
+            ref = oracle_scores(oracle, cache, K, V, Q, b, h).astype(np.float64)
+            rel = np.abs(s_gpu[b, h] - ref) / np.maximum(np.abs(ref), 1e-30)
+            assert rel.max() <= SCORE_RTOL, f"unit {(b, h)}: relative error {rel.max():.3e}"
+    finally:
+        cache.close()
+
+
 def test_full_scores_feed_the_compression(zb, oracle):
     """Scores from the full-history pass, handed to the compression as precomputed scores, give
     the oracle's selection, merge chain and state for a window equal to the prompt."""
