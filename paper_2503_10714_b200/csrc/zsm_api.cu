@@ -7,6 +7,7 @@
 #include <cstring>
 #include <new>
 #include <queue>
+#include <unordered_map>
 #include <vector>
 
 #include "zsm_decode.cuh"
@@ -21,6 +22,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxSmemPerCta = 232448;  // 227 KiB opt-in limit on sm_100
+constexpr int kMaxSmemPerSm = 233472;   // 228 KiB per SM, of which each resident CTA reserves 1 KiB
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
@@ -63,6 +65,25 @@ struct zsm_cache {
     int l_stride, br_max, br_max_pad, cap_max;
     int smem_bytes;
     std::vector<int> layer_cap_max, layer_br_max;
+    // Which layer the last call enqueued on a stream wrote (kWroteAll: every layer).  A per-layer
+    // decode launch may read its layer's cache before the stream's preceding kernel has finished
+    // only if that kernel is known not to write it: the last call on the same stream was this
+    // library's and wrote a different single layer.  (Whatever else the caller put in between
+    // was launched the ordinary way, after our call had completed.)
+    static constexpr int32_t kWroteAll = -1;
+    std::unordered_map<cudaStream_t, int32_t> last_write;
+    void wrote(cudaStream_t s, int32_t layer) {
+        if (last_write.size() > 256) last_write.clear();
+        last_write[s] = layer;
+    }
+    void wrote_everywhere() {
+        for (auto &kv : last_write) kv.second = kWroteAll;
+    }
+    bool may_read_early(cudaStream_t s, int32_t layer) const {
+        if (layer < 0) return false;
+        const auto it = last_write.find(s);
+        return it != last_write.end() && it->second != kWroteAll && it->second != layer;
+    }
 };
 
 namespace {
@@ -388,16 +409,37 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
             for (int C = kSplitMaxCluster; C >= 2 && pl.split == 0; C >>= 1) {
                 if (C > limit || units * C > c->n_sm) continue;
                 const int ls = split_l_stride(c->cap_max, c->br_max, s.esz, C);
-                // merged keys stay in shared memory on rank 0 when they are few (Eq. (hatr))
+                // merged keys stay in shared memory on rank 0 when they are few (Eq. (hatr)) and
+                // the CTA has the SM's shared memory to itself
                 int kr_rows = c->br_max * s.D * 4 <= 32768 ? c->br_max : 0;
                 auto total = [&](int st) {
                     return (int)split_smem_layout(st, s.G, s.D, s.row_bytes, ls, c->br_max_pad,
-                                                  kr_rows, warps).total;
+                                                  kr_rows, warps, C).total;
                 };
-                int st = (kMaxSmemPerCta - total(0) - 64) / (kTileBytes + 16);
-                if (cfg->tune_stages > 0) st = std::min(st, (int)cfg->tune_stages);
-                st = std::min(st, 12);
-                while (st >= 2 && total(st) > kMaxSmemPerCta) --st;
+                auto fit_stages = [&](int budget) {
+                    int n = (budget - total(0) - 64) / (kTileBytes + 16);
+                    n = std::min(n, 12);
+                    while (n >= 2 && total(n) > budget) --n;
+                    return n;
+                };
+                // Two CTAs of this shape fit on an SM when each stays within half of its shared
+                // memory (less the per-CTA reserve): the next layer's launch can then settle in
+                // beside this one's and have its first tiles in flight before this one ends.
+                // Taken when it leaves at least three ring stages; otherwise the whole SM.
+                // (Keeping the merged keys out of shared memory to gain a stage loses: the tail
+                // warp's reads of them are then the last thing the launch waits for; c4 14.9 ->
+                // 16.4 us per layer.)
+                const int pair_budget = kMaxSmemPerSm / 2 - 1024 - 256;
+                int st = 0;
+                if (warps <= kPairConsumerWarps && (cfg->tune_stages == 0 || cfg->tune_stages <= 7)) {
+                    st = fit_stages(pair_budget);
+                    if (cfg->tune_stages > 0) st = std::min(st, (int)cfg->tune_stages);
+                    if (st < 3) st = 0;
+                }
+                if (st == 0) {
+                    st = fit_stages(kMaxSmemPerCta);
+                    if (cfg->tune_stages > 0) st = std::min(st, (int)cfg->tune_stages);
+                }
                 if (st < 2) continue;
                 int fit = 0;
                 const int rc = prepare_decode_split(s.dtype, s.D, s.G, C, total(st),
@@ -468,6 +510,7 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
 
 zsm_status_t zsm_cache_reset(zsm_cache_t *c, zsm_stream_t stream) {
     if (!c) return ZSM_ERR_INVALID_ARG;
+    c->wrote(static_cast<cudaStream_t>(stream), zsm_cache::kWroteAll);
     return cuda_status(cudaMemsetAsync(c->base + c->lay.counters, 0,
                                        (size_t)c->s.n_units * sizeof(UnitCounters),
                                        static_cast<cudaStream_t>(stream)));
@@ -549,11 +592,14 @@ zsm_status_t zsm_decode_step(zsm_cache_t *c, int32_t layer, const void *q, const
         sp.d.l_stride = pl.split_l_stride;
         sp.n_units = layer < 0 ? c->s.n_units : c->s.upl;
         sp.kr_rows = pl.split_kr_rows;
+        sp.early = c->may_read_early(static_cast<cudaStream_t>(stream), layer) ? 1 : 0;
+        c->wrote(static_cast<cudaStream_t>(stream), layer < 0 ? zsm_cache::kWroteAll : layer);
         const int rs = launch_decode_split(c->s.dtype, c->s.D, c->s.G, sp, pl.split, pl.split_warps,
                                            static_cast<cudaStream_t>(stream));
         if (rs == -1) return ZSM_ERR_UNSUPPORTED;
         return rs == 0 ? ZSM_OK : ZSM_ERR_CUDA;
     }
+    c->wrote(static_cast<cudaStream_t>(stream), layer < 0 ? zsm_cache::kWroteAll : layer);
     const int rc = launch_decode_fused(c->s.dtype, c->s.D, c->s.G, p, pl.grid, pl.consumer_warps,
                                        pl.wide, static_cast<cudaStream_t>(stream));
     if (rc == -1) return ZSM_ERR_UNSUPPORTED;
@@ -639,6 +685,7 @@ zsm_status_t zsm_prefill_compress(zsm_cache_t *c, int32_t layer, const void *K, 
     p.cosine = c->cosine;
     p.lambda = c->lambda;
     p.scale = c->scale;
+    c->wrote(static_cast<cudaStream_t>(stream), layer);
     const int rc = launch_prefill(c->s.dtype, c->s.D, p, std::max(1, c->layer_br_max[layer]),
                                   static_cast<cudaStream_t>(stream));
     if (rc == -1) return ZSM_ERR_UNSUPPORTED;
@@ -751,6 +798,7 @@ zsm_status_t zsm_cache_import_unit(zsm_cache_t *c, int32_t layer, int32_t b, int
         if (std::isnan(score[i])) return ZSM_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaStreamSynchronize(cs) != cudaSuccess) return ZSM_ERR_CUDA;
+    c->wrote_everywhere();
     std::vector<uint8_t> raw(cap * s.row_bytes);
     cudaError_t e = cudaSuccess;
     for (int which = 0; which < 2 && e == cudaSuccess; ++which) {

@@ -14,6 +14,15 @@
 // the same time instead of all warps sharing one.  All cross-CTA waits are on mbarriers with a
 // time limit; the cluster barrier at the end keeps a CTA's shared memory alive until its peers
 // are done with it.
+//
+// The launch is a programmatic dependent launch: barrier set-up, the cluster barrier and (when
+// the caller's stream order allows it, SplitParams::early) the unit's counters and a ring-full of
+// K tiles are taken care of while the preceding kernel of the stream is still running; only then
+// does the kernel wait for that kernel (griddepcontrol.wait) and fetch what depends on it -- q,
+// k_new, v_new and the fusion counts, into a header buffer of their own.  It lets its own
+// successor start (griddepcontrol.launch_dependents) right after that wait, never before, so at
+// most two kernels of a stream overlap.  A CTA is sized so that two fit on an SM: the next
+// layer's CTAs settle in beside this layer's.
 #include "zsm_decode_split.cuh"
 
 #include <type_traits>
@@ -23,12 +32,14 @@ namespace zsm {
 namespace {
 
 constexpr int kSplitThreads = (kMaxConsumerWarps + kExtraWarps) * 32;
+constexpr int kSplitPairThreads = (kPairConsumerWarps + kExtraWarps) * 32;
 constexpr int kSplitMaxDynamicSmem = 232448;  // 227 KiB, the opt-in limit per CTA on sm_100
 constexpr int kSplitVGroup = 2;
 
 enum : int32_t {
     WS_PRODUCER = 21, WS_HEADER = 22, WS_K = 23, WS_KR = 24, WS_META = 25, WS_V = 26, WS_VR = 27,
-    WS_SOFTMAX = 28, WS_VICTIM = 29, WS_DONE_OUT = 30, WS_DONE_TAIL = 31, WS_VICTIM_LOCAL = 32
+    WS_SOFTMAX = 28, WS_VICTIM = 29, WS_DONE_OUT = 30, WS_DONE_TAIL = 31, WS_VICTIM_LOCAL = 32,
+    WS_HEADER_TAIL = 33
 };
 
 struct __align__(16) VictimPost {
@@ -70,9 +81,24 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t ra) {
 __device__ __forceinline__ void fence_cluster() {
     asm volatile("fence.acq_rel.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void cluster_sync_all() {
+__device__ __forceinline__ void cluster_arrive() {
     asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
     asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    cluster_arrive();
+    cluster_wait();
+}
+// Programmatic dependent launch: wait until the kernels this launch depends on have completed
+// and their writes are visible (returns at once for an ordinary launch) ...
+__device__ __forceinline__ void griddep_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+// ... and let the next kernel of the stream begin its own prologue.
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity, uint32_t hint_ns) {
     uint32_t ok;
@@ -148,8 +174,7 @@ __device__ __forceinline__ void load4s(const T *p, float (&f)[4]) {
 // when its role is done or a bounded wait gave up; it never leaves the kernel from here.
 template <typename T, int D, int G>
 __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem, const SplitSmem &L,
-                                           const UnitDesc &d, const int4 cnt, const int rank,
-                                           const int C) {
+                                           const UnitDesc &d, const int rank, const int C) {
     using E = Elem<T>;
     const DecodeParams &p = sp.d;
     constexpr int EPL = E::EPL;
@@ -182,14 +207,15 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     uint64_t *x_vict = x_soft + 1;     // rank 0's: every rank's victim candidate is in
     uint64_t *x_done = x_vict + 1;     // rank 0's: partial outputs in, last tiles read
     uint64_t *l_vict = x_done + 1;     // own consumer warps -> tail warp: candidates are in
+    uint64_t *hdr_bar = l_vict + 1;    // the header (q, k_new, v_new, fusion counts) has landed
     volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(smem + L.flags);
     float *probs = reinterpret_cast<float *>(smem + L.probs);  // [local slot][G]
     float *qf = reinterpret_cast<float *>(smem + L.qf);
-    uint8_t *mailp = smem + L.mail;
-    float *s_tok_box = reinterpret_cast<float *>(mailp);
-    uint4 *kn_raw = reinterpret_cast<uint4 *>(mailp + kMailFixed);
-    uint4 *vn_raw = reinterpret_cast<uint4 *>(mailp + kMailFixed + ROWB);
-    uint32_t *w_s = reinterpret_cast<uint32_t *>(mailp + kMailFixed + 2 * ROWB);
+    const uint8_t *hdr = smem + L.hdr;
+    float *s_tok_box = reinterpret_cast<float *>(smem + L.mail);
+    const uint4 *kn_raw = reinterpret_cast<const uint4 *>(hdr + HDR_K);
+    const uint4 *vn_raw = reinterpret_cast<const uint4 *>(hdr + HDR_V);
+    const uint32_t *w_s = reinterpret_cast<const uint32_t *>(hdr + HDR_W);
     float *krs = reinterpret_cast<float *>(smem + L.krs);
     float *opart = reinterpret_cast<float *>(smem + L.opart);
     float *redf = reinterpret_cast<float *>(smem + L.redf);
@@ -202,7 +228,15 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
+    const bool is_producer = warp == NW && lane == 0;
 
+    // Every peer's barriers exist once the cluster barrier of the prologue completes; the
+    // producer thread needs only this CTA's own and passes it after its first copies are out.
+    if (!is_producer) cluster_wait();
+    // The unit's counters were written by this unit's previous step.  With `early` the caller's
+    // stream order guarantees that step finished long ago; otherwise wait for the predecessor.
+    if (!sp.early) griddep_wait();
+    const int4 cnt = *reinterpret_cast<const int4 *>(p.counters + d.unit);
     const int cap = d.Bp + d.Bc;
     const int n_live = min(max(cnt.x, 0), cap);
     const int n_res = min(max(cnt.y, 0), d.Br);
@@ -223,7 +257,33 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
         int s = 0;
         uint32_t ph = 0;
         bool ok = true;
+        // The header depends on the preceding kernel (q, k_new, v_new are its results; the
+        // fusion counts may be): it is requested after the dependency wait.  With `early` up to a
+        // ring-full of tiles is requested before that wait.
+        bool header_out = false;
+        int issued = 0;
+        auto header = [&]() {
+            if (sp.early) {
+                cluster_wait();
+                griddep_wait();
+            }
+            griddep_launch_dependents();
+            mbar_arrive_expect_tx(hdr_bar, HDR_W + br_pad * 4u);
+            uint8_t *dst = smem + L.hdr;
+            bulk_g2s(dst, static_cast<const uint8_t *>(p.q) + (size_t)ul * G * ROWB, G * ROWB, hdr_bar);
+            bulk_g2s(dst + HDR_K, static_cast<const uint8_t *>(p.k_new) + (size_t)ul * ROWB, ROWB, hdr_bar);
+            bulk_g2s(dst + HDR_V, static_cast<const uint8_t *>(p.v_new) + (size_t)ul * ROWB, ROWB, hdr_bar);
+            if (br_pad > 0) bulk_g2s(dst + HDR_W, p.base + d.w_off, br_pad * 4u, hdr_bar);
+            header_out = true;
+        };
+        if (!sp.early) {
+            cluster_wait();
+            header();
+        }
         auto acquire = [&](uint32_t bytes, uint64_t *&bar) -> uint8_t * {
+            // the consumers free no stage before they have the header: once the ring is full
+            // the header has to go out first
+            if (!header_out && issued == S) header();
             if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, p.status, WS_PRODUCER)) {
                 ok = false;
                 return nullptr;
@@ -235,16 +295,11 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
                 s = 0;
                 ph ^= 1u;
             }
+            ++issued;
             return dst;
         };
         uint64_t *bar = nullptr;
-        uint8_t *dst = acquire(HDR_W + br_pad * 4u, bar);
-        if (ok) {
-            bulk_g2s(dst, static_cast<const uint8_t *>(p.q) + (size_t)ul * G * ROWB, G * ROWB, bar);
-            bulk_g2s(dst + HDR_K, static_cast<const uint8_t *>(p.k_new) + (size_t)ul * ROWB, ROWB, bar);
-            bulk_g2s(dst + HDR_V, static_cast<const uint8_t *>(p.v_new) + (size_t)ul * ROWB, ROWB, bar);
-            if (br_pad > 0) bulk_g2s(dst + HDR_W, p.base + d.w_off, br_pad * 4u, bar);
-        }
+        uint8_t *dst;
         // merged keys first: they are few, and their logits need a logarithm each
         for (int r0 = 0; r0 < nr_loc && ok; r0 += R32) {
             const uint32_t bytes = static_cast<uint32_t>(min(R32, nr_loc - r0)) * ROWB32;
@@ -274,6 +329,7 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
             dst = acquire(bytes, bar);
             if (ok) bulk_g2s(dst, p.base + d.vr_off + (size_t)r0 * ROWB32, bytes, bar);
         }
+        if (!header_out) header();  // a unit shorter than the ring
         if (!ok) {
             // give copies already in flight time to land before the CTA's memory goes away
             const uint64_t t0 = global_timer_ns();
@@ -281,6 +337,10 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
         }
         return;
     }
+    // every other thread: nothing below may run before the preceding kernel is complete, except
+    // the tail warp's prefetch of the merged keys when `early` allows it
+    const bool is_tail = warp == NW + 1;
+    if (sp.early && !is_tail) griddep_wait();
 
     const int l32 = lane % LPR32;  // 16-byte column of an fp32 residual row
     const int sub32 = lane / LPR32;
@@ -302,6 +362,7 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
                              : "memory");
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
+        if (sp.early) griddep_wait();
         // this rank's candidate: the lowest of its consumer warps', posted to rank 0
         if (!mbar_wait_bounded(l_vict, 0, abort_flag, p.status, WS_VICTIM_LOCAL)) {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -323,7 +384,8 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
             }
         }
         if (rank != 0) return;
-        if (!mbar_wait_bounded_cluster(x_vict, 0, abort_flag, p.status, WS_VICTIM)) {
+        if (!mbar_wait_bounded_cluster(x_vict, 0, abort_flag, p.status, WS_VICTIM) ||
+            !mbar_wait_bounded(hdr_bar, 0, abort_flag, p.status, WS_HEADER_TAIL)) {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             return;
         }
@@ -513,8 +575,8 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
         dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 1);
 
     // ---------------- header ----------------
-    const uint8_t *h = wait_full(WS_HEADER);
-    if (!h) return;
+    if (!mbar_wait_bounded(hdr_bar, 0, abort_flag, p.status, WS_HEADER)) return;
+    const uint8_t *h = hdr;
     uint32_t qb[kMma ? SEG : 1][4];  // B fragments of q: head n = lane / 4; heads >= G are zero
     if constexpr (kMma) {
         const int gq = lane >> 2, tig = lane & 3;
@@ -531,17 +593,8 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     {
         const T *qs = reinterpret_cast<const T *>(h);
         for (int k = tid; k < G * D; k += NT) qf[k] = E::to_float(qs[k]);
-        const uint4 *ks = reinterpret_cast<const uint4 *>(h + HDR_K);
-        const uint4 *vs = reinterpret_cast<const uint4 *>(h + HDR_V);
-        for (int k = tid; k < ROWB / 16; k += NT) {
-            kn_raw[k] = ks[k];
-            vn_raw[k] = vs[k];
-        }
-        const uint32_t *ws = reinterpret_cast<const uint32_t *>(h + HDR_W);
-        for (int k = tid; k < br_pad; k += NT) w_s[k] = ws[k];
     }
-    release();
-    csync();  // qf and the mailbox arrays are in place
+    csync();  // qf is in place
 
     // ---------------- D1: logits of the merged slots, + alpha ln w (rank 0) ----------------
     for (int r0 = 0; r0 < nr_loc; r0 += R32) {
@@ -897,8 +950,11 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     }
 }
 
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kSplitThreads, 1) decode_split_kernel(const SplitParams sp) {
+// TWO: launch bounds for two CTAs of ten warps per SM (the default shape); otherwise one CTA of up
+// to eighteen warps.
+template <typename T, int D, int G, bool TWO>
+__global__ void __launch_bounds__(TWO ? kSplitPairThreads : kSplitThreads, TWO ? 2 : 1)
+    decode_split_kernel(const SplitParams sp) {
     extern __shared__ __align__(128) uint8_t smem[];
     const DecodeParams &p = sp.d;
     const int NW = (blockDim.x >> 5) - kExtraWarps;
@@ -906,8 +962,8 @@ __global__ void __launch_bounds__(kSplitThreads, 1) decode_split_kernel(const Sp
     const int rank = static_cast<int>(cluster_ctarank());
     const int ci = blockIdx.x / C;  // the cluster's unit, in the launch's plain order
     const SplitSmem L = split_smem_layout(p.stages, G, D, D * (int)sizeof(T), p.l_stride,
-                                          p.br_max_pad, sp.kr_rows, NW);
-    // descriptor and counters straight from global memory, in flight across the set-up below
+                                          p.br_max_pad, sp.kr_rows, NW, C);
+    // the descriptor table is written once, when the cache is created: safe to read at any time
     UnitDesc d;
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(p.sched_desc + ci);
@@ -915,7 +971,6 @@ __global__ void __launch_bounds__(kSplitThreads, 1) decode_split_kernel(const Sp
 #pragma unroll
         for (int k = 0; k < 5; ++k) dst[k] = __ldg(src + k);
     }
-    const int4 cnt = *reinterpret_cast<const int4 *>(p.counters + p.unit_base + ci);
 
     if (threadIdx.x == 0) {
         uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
@@ -929,16 +984,24 @@ __global__ void __launch_bounds__(kSplitThreads, 1) decode_split_kernel(const Sp
         // partial outputs, last tiles read (used on rank 0): every posting warp of every rank
         mbar_init(&bars[2 * S + 2], C * split_post_warps(NW, G * D));
         mbar_init(&bars[2 * S + 3], NW);  // victim candidates of this CTA's consumer warps
+        mbar_init(&bars[2 * S + 4], 1);   // header
         *reinterpret_cast<volatile int32_t *>(smem + L.flags) = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    cluster_sync_all();  // every peer's barriers exist before anything is posted to them
+    // First cluster barrier: every peer's barriers exist before anything is posted to them.
+    // Each thread completes it (cluster_wait) where its role first needs it, in split_body.
+    cluster_arrive();
     if (d.unit == p.unit_base + ci) {
-        split_body<T, D, G>(sp, smem, L, d, cnt, rank, C);
-    } else if (threadIdx.x == 0 && rank == 0) {
-        dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 3);
+        split_body<T, D, G>(sp, smem, L, d, rank, C);
+    } else {
+        cluster_wait();
+        if (threadIdx.x == 0) {
+            griddep_wait();
+            griddep_launch_dependents();
+            if (rank == 0) dev_set_status(p.status, DEV_ERR_CHECK, d.unit, 3);
+        }
     }
     cluster_sync_all();  // no CTA leaves while a peer may still write to its shared memory
 }
@@ -948,25 +1011,30 @@ int launch_split_one(const SplitParams &sp, int cluster, int consumer_warps, cud
     const DecodeParams &p = sp.d;
     const int threads = (consumer_warps + kExtraWarps) * 32;
     const SplitSmem L = split_smem_layout(p.stages, G, D, D * (int)sizeof(T), p.l_stride,
-                                          p.br_max_pad, sp.kr_rows, consumer_warps);
+                                          p.br_max_pad, sp.kr_rows, consumer_warps, cluster);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(sp.n_units * cluster), 1, 1);
     cfg.blockDim = dim3(static_cast<unsigned>(threads), 1, 1);
     cfg.dynamicSmemBytes = L.total;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // the kernel orders itself after its predecessor with griddepcontrol.wait
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return static_cast<int>(cudaLaunchKernelEx(&cfg, decode_split_kernel<T, D, G>, sp));
+    cfg.numAttrs = 2;
+    if (threads <= kSplitPairThreads)
+        return static_cast<int>(cudaLaunchKernelEx(&cfg, decode_split_kernel<T, D, G, true>, sp));
+    return static_cast<int>(cudaLaunchKernelEx(&cfg, decode_split_kernel<T, D, G, false>, sp));
 }
 
-template <typename T, int D, int G>
-int prepare_split_one(int cluster, int smem_bytes, int threads, int *max_clusters) {
-    cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<T, D, G>,
+template <typename T, int D, int G, bool TWO>
+int prepare_split_form(int cluster, int smem_bytes, int threads, int *max_clusters) {
+    cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<T, D, G, TWO>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kSplitMaxDynamicSmem);
     if (e != cudaSuccess) return static_cast<int>(e);
@@ -982,9 +1050,16 @@ int prepare_split_one(int cluster, int smem_bytes, int threads, int *max_cluster
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, decode_split_kernel<T, D, G>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, decode_split_kernel<T, D, G, TWO>, &cfg);
     if (max_clusters) *max_clusters = n;
     return static_cast<int>(e);
+}
+
+template <typename T, int D, int G>
+int prepare_split_one(int cluster, int smem_bytes, int threads, int *max_clusters) {
+    if (threads <= kSplitPairThreads)
+        return prepare_split_form<T, D, G, true>(cluster, smem_bytes, threads, max_clusters);
+    return prepare_split_form<T, D, G, false>(cluster, smem_bytes, threads, max_clusters);
 }
 
 #define ZSM_SPLIT_DISPATCH(FN, ...)                                                   \

@@ -16,6 +16,9 @@ struct SplitParams {
                           // l_stride: weight entries one CTA can hold (split_l_stride)
     int32_t n_units;      // clusters in the launch
     int32_t kr_rows;      // merged key rows rank 0 can keep in shared memory (0: none)
+    int32_t early;        // 1: the kernel that precedes this launch in its stream does not write
+                          // these units' cache, so their counters and first tiles may be read
+                          // while that kernel is still running (programmatic dependent launch)
 };
 
 // Token rows [lo, hi) of rank c of C.  Rank 0 also carries the merged rows (fp32 masters, so one
@@ -60,12 +63,18 @@ __host__ __device__ inline int split_l_stride(int cap_max, int br_max, int elem_
 
 // Shared-memory map of one CTA of the split form (byte offsets).
 struct SplitSmem {
-    uint32_t ring, bars, flags, probs, qf, mail, krs, opart, redf, red64, xs, xv, xo, total;
+    uint32_t ring, bars, flags, hdr, probs, qf, mail, krs, opart, redf, red64, xs, xv, xo, total;
 };
+
+// Bytes of the header a CTA receives after the launch's inputs are known to be ready: q (G rows),
+// k_new, v_new in the storage dtype, then the unit's fusion counts.
+__host__ __device__ inline uint32_t split_header_bytes(int G, int row_bytes, int br_max_pad) {
+    return static_cast<uint32_t>((G + 2) * row_bytes + br_max_pad * 4);
+}
 
 __host__ __device__ inline SplitSmem split_smem_layout(int stages, int G, int D, int row_bytes,
                                                        int l_stride, int br_max_pad, int kr_rows,
-                                                       int consumer_warps) {
+                                                       int consumer_warps, int cluster) {
     SplitSmem L;
     uint32_t o = 0;
     auto take = [&](uint32_t bytes) {
@@ -74,8 +83,9 @@ __host__ __device__ inline SplitSmem split_smem_layout(int stages, int G, int D,
         return at;
     };
     L.ring = take(static_cast<uint32_t>(stages) * kTileBytes);
-    L.bars = take((2u * static_cast<uint32_t>(stages) + 4u) * 8u);
+    L.bars = take((2u * static_cast<uint32_t>(stages) + 5u) * 8u);
     L.flags = take(64u);
+    L.hdr = take(split_header_bytes(G, row_bytes, br_max_pad));
     L.probs = take(static_cast<uint32_t>(G) * l_stride * 4u);
     L.qf = take(static_cast<uint32_t>(G) * D * 4u);
     L.mail = take(decode_mail_bytes(row_bytes, br_max_pad));
@@ -85,7 +95,7 @@ __host__ __device__ inline SplitSmem split_smem_layout(int stages, int G, int D,
     L.red64 = take(kMaxConsumerWarps * 16u);
     L.xs = take(kSplitMaxCluster * 2u * 8u * 4u);                       // (max, sum) per rank and head
     L.xv = take(kSplitMaxCluster * 16u);                                // victim candidate per rank
-    L.xo = take(kSplitMaxCluster * static_cast<uint32_t>(G) * D * 4u);  // partial outputs per rank
+    L.xo = take(static_cast<uint32_t>(cluster) * G * D * 4u);           // partial outputs per rank
     L.total = o;
     return L;
 }
