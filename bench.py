@@ -12,6 +12,12 @@ far larger than L2, so no flush is needed between steps).
 N > 1 (torchrun): every rank runs the same workload on its own sequence (weak scaling,
 no data-path collective); value = tokens of all ranks / max-over-ranks device time.
 
+The timed region is repeated (--repeats, default 5): `ms_per_step` is the median of the
+repeats' CUDA-event times, `spread` their (max - min) / median; SM clocks are sampled every
+millisecond and reported per repeat.  At N = 1 the other named workloads (c3, c4 at 10 % and
+20 %, c5) are run after the headline one and reported under `configs`, each with its own
+roofline and clocks (--configs none skips them).
+
 --impl reference times the CPU oracle (the only other implementation of this path that
 exists) on a bounded sample of the same workload, rank 0 only.
 """
@@ -79,13 +85,15 @@ def recorded_traffic(w):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML every millisecond, each sample with
+    its host time, so that a window of the run (one repeat of the timed region) can be
+    summarised by itself."""
 
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
                0x4: "sw_power_cap", 0x80: "hw_power_brake"}
 
     def __init__(self, index):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.max_mhz = [], None   # (host time, MHz, reason mask)
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -100,14 +108,12 @@ class ClockSampler:
     def _run(self):
         while not self._stop.is_set():
             try:
-                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                mhz = self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)
                 mask = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
-                for bit, name in self.REASONS.items():
-                    if mask & bit:
-                        self.reasons.add(name)
+                self.samples.append((time.perf_counter(), mhz, mask))
             except Exception:
                 pass
-            time.sleep(0.01)
+            time.sleep(0.001)
 
     def __enter__(self):
         if self.nv:
@@ -120,10 +126,45 @@ class ClockSampler:
         if self._thread:
             self._thread.join()
 
-    def summary(self):
-        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+    def summary(self, windows=None):
+        """Median SM MHz and the reasons seen, over the given (t0, t1) host-time windows (all
+        samples when None); `per_repeat` lists each window's own median."""
+        def inside(t):
+            return windows is None or any(a <= t <= b for a, b in windows)
+        sel = [(m, k) for t, m, k in self.samples if inside(t)]
+        reasons = sorted({name for _, k in sel for bit, name in self.REASONS.items() if k & bit})
+        out = {"sm_mhz": float(np.median([m for m, _ in sel])) if sel else None,
+               "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(sel),
+               "period_ms": 1}
+        if windows is not None:
+            per = []
+            for a, b in windows:
+                ms = [m for t, m, _ in self.samples if a <= t <= b]
+                per.append(float(np.median(ms)) if ms else None)
+            out["per_repeat_sm_mhz"] = per
+        return out
+
+
+NOMINAL_HBM_GBS = 8000.0   # the figure the 70 % target is stated against
+
+
+def parity_counts(workload_name):
+    """Near-tie / exact-tie counts of the full-size parity tests for this workload, from the
+    kept record profiles/parity_counts.md (JSON lines written by tests/test_gpu_full_size.py)."""
+    out = []
+    try:
+        with open(os.path.join(ROOT, "profiles", "parity_counts.md")) as f:
+            for line in f:
+                line = line.strip()
+                if line.startswith("{"):
+                    rec = json.loads(line)
+                    if rec.get("workload") == workload_name:
+                        out.append({k: rec[k] for k in ("launches", "sampled_units", "steps", "selections",
+                                                         "merges", "victim_near_ties", "merge_near_ties",
+                                                         "exact_tie_breaches") if k in rec})
+    except Exception:
+        return None
+    return out or None
 
 
 def algorithmic_bytes(w, bp, bc, br, n_live, n_res):
@@ -347,14 +388,256 @@ def measured_tensor_peak():
         return 1590.0
 
 
+# ----------------------------------------------------------------------------- one workload
+def make_budgets(zb, w):
+    totals = wl.head_budgets(w)
+    bp, bc, br = np.zeros_like(totals), np.zeros_like(totals), np.zeros_like(totals)
+    for idx in np.ndindex(totals.shape):
+        bp[idx], bc[idx], br[idx] = zb.zsm_split_budget(int(totals[idx]))
+    return totals, bp, bc, br
+
+
+def prompt_pass(zb, cache, w, dev, u, stream, keep_layer0):
+    """Every layer's prompt through the real compression kernels, one layer after another on
+    one stream (timed per layer with events).  Returns (ms total, host copy of layer 0's prompt)."""
+    ws = torch.empty(zb.zsm_prefill_workspace_bytes(cache, w.prompt_len, w.window),
+                     dtype=torch.uint8, device=dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    total, sample = 0.0, None
+    for layer in range(w.n_layers):
+        Kp, Vp, Qw = wl.prompt(w, layer, dev, u)
+        ev0.record(stream)
+        zb.zsm_prefill_compress(cache, layer, Kp, Vp, Qw, None, w.prompt_len, w.window, ws)
+        ev1.record(stream)
+        ev1.synchronize()
+        total += ev0.elapsed_time(ev1)
+        if layer == 0 and keep_layer0:
+            sample = (Kp.cpu(), Vp.cpu(), Qw.cpu())
+        del Kp, Vp, Qw
+    del ws
+    torch.cuda.empty_cache()
+    if zb.zsm_last_device_status(cache) != 0:
+        raise RuntimeError("device status after the prompt pass is not OK")
+    return total, sample
+
+
+def prompt_pass_overlapped(zb, cache, w, dev, u, n_streams=4, n_layers=8):
+    """The prompt pass of `n_layers` layers issued round-robin on `n_streams` streams, each with
+    its own workspace: the residual chain of one layer occupies one CTA per unit (32 of 148 SMs
+    at c4), so several layers' chains run side by side.  Prompts are generated beforehand; the
+    time is wall-to-wall device time over all streams, per layer."""
+    per_layer_bytes = 2 * w.batch * w.n_kv_heads * w.prompt_len * w.head_dim * (4 if w.dtype == "f32" else 2)
+    n_layers = int(min(n_layers, w.n_layers, max(2, 30e9 // per_layer_bytes)))
+    n_streams = min(n_streams, n_layers)
+    need = zb.zsm_prefill_workspace_bytes(cache, w.prompt_len, w.window)
+    wss = [torch.empty(need, dtype=torch.uint8, device=dev) for _ in range(n_streams)]
+    streams = [torch.cuda.Stream(device=dev) for _ in range(n_streams)]
+    prompts = [wl.prompt(w, layer, dev, u) for layer in range(n_layers)]
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    main = torch.cuda.current_stream()
+    ev0.record(main)
+    for st in streams:
+        st.wait_event(ev0)
+    for layer in range(n_layers):
+        st = streams[layer % n_streams]
+        Kp, Vp, Qw = prompts[layer]
+        zb.zsm_prefill_compress(cache, layer, Kp, Vp, Qw, None, w.prompt_len, w.window,
+                                wss[layer % n_streams], stream=st)
+    for st in streams:
+        main.wait_stream(st)
+    ev1.record(main)
+    ev1.synchronize()
+    if zb.zsm_last_device_status(cache) != 0:
+        raise RuntimeError("device status after the overlapped prompt pass is not OK")
+    ms = ev0.elapsed_time(ev1)
+    del prompts, wss
+    torch.cuda.empty_cache()
+    return {"what": "%d layers round-robin on %d streams, one workspace per stream" % (n_layers, n_streams),
+            "layers": n_layers, "streams": n_streams, "ms_per_layer": ms / n_layers,
+            "ms_total_scaled": ms / n_layers * w.n_layers}
+
+
+def run_workload(zb, w, args, dev, local, world, rank, headline):
+    """Prompt pass, then the timed decode steps of one workload.  Returns the result dict (on
+    every rank; only rank 0's is printed)."""
+    stream = torch.cuda.current_stream()
+    totals, bp, bc, br = make_budgets(zb, w)
+    W, K, R = max(3, args.warmup), max(1, args.steps), max(1, args.repeats)
+    cfg = zb.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, bp,
+                         bc, br, tune_stages=args.stages, tune_ctas_per_sm=args.ctas_per_sm,
+                         tune_consumer_warps=args.consumer_warps, tune_split=args.split)
+    buf = torch.empty(zb.zsm_cache_bytes(cfg), dtype=torch.uint8, device=dev)
+    cache = zb.zsm_cache_create(cfg, buf)
+    u = wl.directions(w, dev)
+    want_cpu = headline and rank == 0 and world == 1 and not args.no_cpu_baseline
+    prefill_ms, sample_prompt = prompt_pass(zb, cache, w, dev, u, stream, want_cpu)
+
+    # ---- decode inputs for every step, resident in HBM before timing starts ----
+    n_in = W + K
+    qs = torch.empty(n_in, w.n_layers, w.batch, w.n_q_heads, w.head_dim, dtype=w.torch_dtype, device=dev)
+    ks = torch.empty(n_in, w.n_layers, w.batch, w.n_kv_heads, w.head_dim, dtype=w.torch_dtype, device=dev)
+    vs = torch.empty_like(ks)
+    for s in range(n_in):
+        qs[s], ks[s], vs[s] = wl.decode_inputs(w, s, dev, u)
+    out = torch.empty_like(qs[0])
+    for s in range(W):
+        zb.zsm_decode_step(cache, -1, qs[s], ks[s], vs[s], out)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rep_ms, windows = [], []
+    with ClockSampler(local) as clocks:
+        for r in range(R):
+            barrier(world)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            ev0.record(stream)
+            for s in range(W, W + K):   # the same K inputs each repeat; the cache keeps evolving
+                zb.zsm_decode_step(cache, -1, qs[s], ks[s], vs[s], out)
+            ev1.record(stream)
+            ev1.synchronize()
+            torch.cuda.synchronize()
+            windows.append((t0, time.perf_counter()))
+            barrier(world)
+            rep_ms.append(max_over_ranks(ev0.elapsed_time(ev1), world))
+    ms_total = float(np.median(rep_ms))
+    ms_per_step = ms_total / K
+    value = world * w.batch * K / (ms_total * 1e-3)
+    spread = (max(rep_ms) - min(rep_ms)) / ms_total
+    if zb.zsm_last_device_status(cache) != 0:
+        raise RuntimeError("device status after the timed region is not OK")
+
+    # ---- roofline of the dominant (only) kernel of the timed region ----
+    n_live = np.minimum((bp + bc).astype(np.int64), w.prompt_len + W)
+    n_res = br.astype(np.int64)
+    abytes = algorithmic_bytes(w, bp, bc, br, n_live, n_res)
+    peak, peak_kind = measured_peak()
+    achieved = abytes / (ms_per_step * 1e-3) / 1e9
+    grid, block, smem = zb.zsm_decode_launch_info(cache, -1)
+    res = {
+        "value": value, "ms_per_step": ms_per_step, "repeats": R, "spread": spread,
+        "ms_per_step_repeats": [m / K for m in rep_ms],
+        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch,
+                   "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                   "prompt_len": w.prompt_len, "slots_per_head": int(totals.mean()),
+                   "launch": "one fused kernel over all layers per step",
+                   "grid": grid, "block": block, "smem_bytes": smem,
+                   "l2": "inputs larger than L2 (%.2f GB streamed per step)" % (abytes / 1e9)},
+        "clocks": clocks.summary(windows),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth of this pool",
+                     "frac_nominal": achieved / NOMINAL_HBM_GBS, "peak_nominal": NOMINAL_HBM_GBS,
+                     "algorithmic_bytes_per_launch": abytes, "traffic": recorded_traffic(w)},
+        "prompt_pass": {"ms_total": prefill_ms, "ms_per_layer": prefill_ms / w.n_layers,
+                        "window": w.window, "what": "layers one after another on one stream"},
+        "dtype": w.dtype,
+    }
+    pc = parity_counts(w.name.split("_%dlayers" % w.n_layers)[0])
+    if pc is not None:
+        res["parity_counts"] = pc
+
+    # ---- the same metric through host buffers (copies inside the timed region) ----
+    if headline:
+        Ke = max(1, min(args.e2e_steps, K))
+        q_off, k_off, v_off, in_bytes, out_bytes = zb.zsm_decode_host_layout(cache, -1)
+        half = in_bytes + (out_bytes + 255) // 256 * 256
+        staging = torch.empty(2 * half, dtype=torch.uint8, device=dev)
+        packed = []
+        for s in range(Ke):
+            t = torch.zeros(in_bytes, dtype=torch.uint8)
+            for off, src in ((q_off, qs[W + s]), (k_off, ks[W + s]), (v_off, vs[W + s])):
+                raw = src.contiguous().view(torch.uint8).reshape(-1).cpu()
+                t[off:off + raw.numel()] = raw
+            packed.append(t.pin_memory())
+        oh = [torch.empty(out.shape, dtype=out.dtype).pin_memory() for _ in range(2)]
+
+        def pipelined(n):
+            for s in range(n + 2):
+                slot = s & 1
+                if s >= 2:
+                    zb.zsm_decode_step_host_wait(cache, slot)
+                if s < n:
+                    zb.zsm_decode_step_host_async(cache, -1, packed[s], oh[slot], staging, slot)
+        pipelined(min(3, Ke))
+        torch.cuda.synchronize()
+        barrier(world)
+        t0 = time.perf_counter()
+        pipelined(Ke)
+        torch.cuda.synchronize()
+        e2e_s = max_over_ranks(time.perf_counter() - t0, world)
+        # and one step at a time: copies in, step, copy out, wait -- nothing overlaps
+        st1 = torch.empty(zb.zsm_decode_staging_bytes(cache, -1), dtype=torch.uint8, device=dev)
+        qh = [qs[W + s].cpu().pin_memory() for s in range(Ke)]
+        kh = [ks[W + s].cpu().pin_memory() for s in range(Ke)]
+        vh = [vs[W + s].cpu().pin_memory() for s in range(Ke)]
+        for s in range(min(3, Ke)):
+            zb.zsm_decode_step_host(cache, -1, qh[s], kh[s], vh[s], oh[0], st1)
+        torch.cuda.synchronize()
+        barrier(world)
+        t0 = time.perf_counter()
+        for s in range(Ke):
+            zb.zsm_decode_step_host(cache, -1, qh[s], kh[s], vh[s], oh[0], st1)
+        torch.cuda.synchronize()
+        sync_s = max_over_ranks(time.perf_counter() - t0, world)
+        res["e2e"] = {"value": world * w.batch * Ke / e2e_s, "unit": "tokens/s",
+                      "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
+                      "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3,
+                      "what": "zsm_decode_step_host_async: pinned host buffers, one copy in and one "
+                              "out per step, two steps in flight",
+                      "one_step_at_a_time": {"value": world * w.batch * Ke / sync_s,
+                                             "ms_per_step": sync_s / Ke * 1e3,
+                                             "what": "zsm_decode_step_host: copies, step, copy, wait"}}
+        del staging, st1, packed, qh, kh, vh
+
+    if rank == 0 and world == 1:
+        # the launch shape a model would use: one launch per layer, the L launches of a step
+        # captured in a CUDA graph (reported beside the headline, not instead of it)
+        if w.n_layers > 1:
+            pl = per_layer_graph(zb, cache, w, qs, ks, vs, out, W, min(K, 200))
+            pl["achieved_gbs"] = abytes / (pl["ms_per_step"] * 1e-3) / 1e9
+            pl["frac"] = pl["achieved_gbs"] / peak
+            res["per_layer_launches"] = pl
+        del qs, ks, vs
+        torch.cuda.empty_cache()
+        if w.n_layers > 1 and not args.no_prompt_overlap:
+            res["prompt_pass"]["overlapped"] = prompt_pass_overlapped(zb, cache, w, dev, u)
+        if headline and not args.no_fullkv and w.dtype != "f32":
+            fk = fullkv_comparator(zb, w, dev, u, stream)
+            fk["compressed_speedup"] = fk["ms_per_step"] / ms_per_step
+            res["fullkv"] = fk
+        if headline and not args.no_full_history and w.dtype != "f32":
+            res["prompt_scores_full_history"] = full_history_scores(zb, cache, w, dev, u, stream)
+        if want_cpu and sample_prompt is not None:
+            dt, n_sampled, threads, dt1 = oracle_sample(w, *sample_prompt, bp, bc, br, args.cpu_steps)
+            n_units = w.n_layers * w.batch * w.n_kv_heads
+            res["cpu_baseline"] = {
+                "value": w.batch / (dt * n_units / n_sampled), "unit": "tokens/s", "cores": threads,
+                "one_thread": w.batch / (dt1 * n_units / n_sampled), "kind": "oracle",
+                "sample": "%d of %d units (layer 0) x %d decode steps, scaled by units" % (
+                    n_sampled, n_units, args.cpu_steps)}
+    zb.zsm_cache_free(cache)
+    del buf
+    torch.cuda.empty_cache()
+    return res
+
+
 # ----------------------------------------------------------------------------- main
+OTHER_CONFIGS = ["c3_llama7b_b16", "c4_54k_10pct", "c4_54k_20pct", "c5_gqa_ragged"]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--repeats", type=int, default=5,
+                    help="times the timed region is run; the median is reported")
     ap.add_argument("--impl", default="zsm", choices=["zsm", "reference"])
     ap.add_argument("--workload", default="c4_54k_5pct", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--configs", default="all", choices=["all", "none"],
+                    help="all: also run the other named workloads (1 GPU only) and report them "
+                         "under `configs`")
+    ap.add_argument("--config-steps", type=int, default=100, help="timed steps of those workloads")
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--cpu-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -362,6 +645,8 @@ def main():
                     help="skip the uncompressed-cache comparator (same box, same shapes)")
     ap.add_argument("--no-full-history", action="store_true",
                     help="skip the full-history (W = T) prompt scoring leg")
+    ap.add_argument("--no-prompt-overlap", action="store_true",
+                    help="skip the prompt pass with layers overlapped on several streams")
     ap.add_argument("--layers", type=int, default=0,
                     help="run a shallower stack than the workload names (profiling captures only; "
                          "the reported config says so)")
@@ -372,173 +657,43 @@ def main():
                     help="CTAs per unit in launches with few units (0: library default, 1: never)")
     args = ap.parse_args()
     world, rank, local = dist_setup(args.gpus)
-    w0 = wl.WORKLOADS[args.workload]
-    W = max(3, args.warmup)
-    K = max(1, args.steps)
-
-    w = rank_workload(w0, rank)
-    if args.layers > 0:
-        w = w.replace(n_layers=args.layers, name=w.name + "_%dlayers" % args.layers)
-    from paper_2503_10714_b200 import binding as zb
-    totals = wl.head_budgets(w)
-    bp = np.zeros_like(totals)
-    bc = np.zeros_like(totals)
-    br = np.zeros_like(totals)
-    for idx in np.ndindex(totals.shape):
-        bp[idx], bc[idx], br[idx] = zb.zsm_split_budget(int(totals[idx]))
-
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    stream = torch.cuda.current_stream()
-    cfg = zb.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, bp,
-                         bc, br, tune_stages=args.stages, tune_ctas_per_sm=args.ctas_per_sm,
-                         tune_consumer_warps=args.consumer_warps, tune_split=args.split)
-    buf = torch.empty(zb.zsm_cache_bytes(cfg), dtype=torch.uint8, device=dev)
-    cache = zb.zsm_cache_create(cfg, buf)
+    from paper_2503_10714_b200 import binding as zb
 
-    # ---- prompt pass (real kernels; timed separately, not part of the decode metric) ----
-    u = wl.directions(w, dev)
-    ws = torch.empty(zb.zsm_prefill_workspace_bytes(cache, w.prompt_len, w.window),
-                     dtype=torch.uint8, device=dev)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    prefill_ms = 0.0
-    sample_prompt = None
-    for layer in range(w.n_layers):
-        Kp, Vp, Qw = wl.prompt(w, layer, dev, u)
-        ev0.record(stream)
-        zb.zsm_prefill_compress(cache, layer, Kp, Vp, Qw, None, w.prompt_len, w.window, ws)
-        ev1.record(stream)
-        ev1.synchronize()
-        prefill_ms += ev0.elapsed_time(ev1)
-        if layer == 0 and rank == 0 and world == 1 and not args.no_cpu_baseline:
-            sample_prompt = (Kp.cpu(), Vp.cpu(), Qw.cpu())
-        del Kp, Vp, Qw
-    del ws
-    torch.cuda.empty_cache()
-    if zb.zsm_last_device_status(cache) != 0:
-        raise RuntimeError("device status after the prompt pass is not OK")
-
-    # ---- decode inputs for every step, resident in HBM before timing starts ----
-    n_steps_total = W + K
-    qs = torch.empty(n_steps_total, w.n_layers, w.batch, w.n_q_heads, w.head_dim,
-                     dtype=w.torch_dtype, device=dev)
-    ks = torch.empty(n_steps_total, w.n_layers, w.batch, w.n_kv_heads, w.head_dim,
-                     dtype=w.torch_dtype, device=dev)
-    vs = torch.empty_like(ks)
-    for s in range(n_steps_total):
-        qs[s], ks[s], vs[s] = wl.decode_inputs(w, s, dev, u)
-    out = torch.empty_like(qs[0])
-    for s in range(W):
-        zb.zsm_decode_step(cache, -1, qs[s], ks[s], vs[s], out)
-    torch.cuda.synchronize()
-    barrier(world)
-    torch.cuda.synchronize()
-    with ClockSampler(local) as clocks:
-        ev0.record(stream)
-        for s in range(W, W + K):
-            zb.zsm_decode_step(cache, -1, qs[s], ks[s], vs[s], out)
-        ev1.record(stream)
-        ev1.synchronize()
-    torch.cuda.synchronize()
-    barrier(world)
-    ms_local = ev0.elapsed_time(ev1)
-    value, ms_total = whole_job_throughput(ms_local, w.batch * K, world)
-    ms_per_step = ms_total / K
-    if zb.zsm_last_device_status(cache) != 0:
-        raise RuntimeError("device status after the timed region is not OK")
-
-    # ---- the same metric through host buffers (copies inside the timed region) ----
-    Ke = max(1, min(args.e2e_steps, K))
-    staging = torch.empty(zb.zsm_decode_staging_bytes(cache, -1), dtype=torch.uint8, device=dev)
-    qh = [qs[W + s].cpu().pin_memory() for s in range(Ke)]
-    kh = [ks[W + s].cpu().pin_memory() for s in range(Ke)]
-    vh = [vs[W + s].cpu().pin_memory() for s in range(Ke)]
-    oh = torch.empty_like(qh[0]).pin_memory()
-    for s in range(min(3, Ke)):
-        zb.zsm_decode_step_host(cache, -1, qh[s], kh[s], vh[s], oh, staging)
-    torch.cuda.synchronize()
-    barrier(world)
-    t0 = time.perf_counter()
-    for s in range(Ke):
-        zb.zsm_decode_step_host(cache, -1, qh[s], kh[s], vh[s], oh, staging)
-    torch.cuda.synchronize()
-    e2e_s = max_over_ranks(time.perf_counter() - t0, world)
-    h2d = qh[0].numel() * qh[0].element_size() + 2 * kh[0].numel() * kh[0].element_size()
-    d2h = oh.numel() * oh.element_size()
-
+    w = rank_workload(wl.WORKLOADS[args.workload], rank)
+    if args.layers > 0:
+        w = w.replace(n_layers=args.layers, name=w.name + "_%dlayers" % args.layers)
+    res = run_workload(zb, w, args, dev, local, world, rank, headline=True)
     if rank != 0:
-        zb.zsm_cache_free(cache)
         return
-
-    # ---- the launch shape a model would use: one launch per layer, the L launches of a step
-    #      captured in a CUDA graph (reported beside the headline, not instead of it) ----
-    per_layer = None
-    if world == 1 and w.n_layers > 1:
-        per_layer = per_layer_graph(zb, cache, w, qs, ks, vs, out, W, min(K, 200))
-
-    fullkv = None
-    if world == 1 and not args.no_fullkv and w.dtype != "f32":
-        fullkv = fullkv_comparator(zb, w, dev, u, stream)
-
-    full_hist = None
-    if world == 1 and not args.no_full_history and w.dtype != "f32":
-        full_hist = full_history_scores(zb, cache, w, dev, u, stream)
-
-    # ---- roofline of the dominant (only) kernel of the timed region ----
-    n_live = (bp + bc).astype(np.int64)      # every unit is full after a 54k prompt
-    n_res = br.astype(np.int64)
-    n_live = np.minimum(n_live, w.prompt_len + W)
-    abytes = algorithmic_bytes(w, bp, bc, br, n_live, n_res)
-    peak, peak_kind = measured_peak()
-    achieved = abytes / (ms_local / K * 1e-3) / 1e9
-    grid, block, smem = zb.zsm_decode_launch_info(cache, -1)
+    K, W = max(1, args.steps), max(3, args.warmup)
     line = {
         "metric": "decode tokens/s with ZSMerge cache update",
-        "value": value,
-        "unit": "tokens/s",
-        "n_gpus": world,
-        "steps": K,
-        "warmup": W,
-        "ms_per_step": ms_per_step,
-        "higher_is_better": True,
-        "scaling": "weak",
-        "vs_baseline": None,
-        "dtype": w.dtype,
-        "data": "synthetic",
-        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch,
-                   "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
-                   "prompt_len": w.prompt_len, "slots_per_head": int(totals.mean()),
-                   "launch": "one fused kernel over all layers per step",
-                   "grid": grid, "block": block, "smem_bytes": smem,
-                   "l2": "inputs larger than L2 (%.2f GB streamed per step)" % (abytes / 1e9)},
-        "clocks": clocks.summary(),
-        "e2e": {"value": world * w.batch * Ke / e2e_s, "unit": "tokens/s",
-                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": Ke},
-        "gpu_launches": K,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": peak_kind,
-                     "algorithmic_bytes_per_launch": abytes,
-                     "traffic": recorded_traffic(w)},
-        "prompt_pass": {"ms_total": prefill_ms, "ms_per_layer": prefill_ms / w.n_layers,
-                        "window": w.window},
+        "value": res["value"], "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": res["ms_per_step"], "repeats": res["repeats"], "spread": res["spread"],
+        "ms_per_step_repeats": res["ms_per_step_repeats"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": res["dtype"],
+        "data": "synthetic", "config": res["config"], "clocks": res["clocks"],
+        "e2e": res.get("e2e"), "gpu_launches": K,
+        "roofline": res["roofline"], "prompt_pass": res["prompt_pass"],
     }
-    if per_layer is not None:
-        line["per_layer_launches"] = per_layer
-    if full_hist is not None:
-        line["prompt_scores_full_history"] = full_hist
-    if fullkv is not None:
-        fullkv["compressed_speedup"] = fullkv["ms_per_step"] / ms_per_step
-        line["fullkv"] = fullkv
-    if world == 1 and not args.no_cpu_baseline and sample_prompt is not None:
-        dt, n_sampled, threads, dt1 = oracle_sample(w, *sample_prompt, bp, bc, br, args.cpu_steps)
-        n_units = w.n_layers * w.batch * w.n_kv_heads
-        line["cpu_baseline"] = {
-            "value": w.batch / (dt * n_units / n_sampled), "unit": "tokens/s", "cores": threads,
-            "one_thread": w.batch / (dt1 * n_units / n_sampled),
-            "kind": "oracle",
-            "sample": "%d of %d units (layer 0) x %d decode steps, scaled by units" % (
-                n_sampled, n_units, args.cpu_steps)}
-    zb.zsm_cache_free(cache)
+    for key in ("parity_counts", "per_layer_launches", "prompt_scores_full_history", "fullkv",
+                "cpu_baseline"):
+        if key in res:
+            line[key] = res[key]
+    if world == 1 and args.configs == "all" and args.layers == 0 and args.workload == "c4_54k_5pct":
+        others = {}
+        sub = argparse.Namespace(**vars(args))
+        sub.steps = max(1, args.config_steps)
+        for name in OTHER_CONFIGS:
+            try:
+                r = run_workload(zb, wl.WORKLOADS[name], sub, dev, local, world, rank, headline=False)
+                r["steps"] = sub.steps
+                others[name] = r
+            except Exception as exc:   # a workload that does not fit must not lose the headline
+                others[name] = {"error": "%s: %s" % (type(exc).__name__, exc)}
+        line["configs"] = others
     print(json.dumps(line))
 
 

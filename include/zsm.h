@@ -237,6 +237,29 @@ zsm_status_t zsm_decode_step_host(zsm_cache_t *c, int32_t layer, const void *q_h
                                   void *out_host, void *staging, size_t staging_bytes,
                                   zsm_stream_t stream);
 
+/* The host-buffer step pipelined over two staging halves, for callers that stream steps: the
+ * call only enqueues -- one copy in on an internal copy stream, the step on `stream`, one copy
+ * out on a second internal copy stream, tied together by events -- and returns; step i+1's
+ * copy in and step i's copy out then run under the other step's kernel.  Steps stay ordered
+ * (they update one cache) because all of them run on `stream`.
+ *   in_host    pinned host buffer holding q, k_new and v_new at the offsets
+ *              zsm_decode_host_layout gives (in_bytes long; one copy moves it)
+ *   out_host   pinned host buffer of out_bytes; valid after zsm_decode_step_host_wait(slot)
+ *   staging    dev scratch, 256-byte aligned, >= 2 * (in_bytes + out_bytes rounded up to 256)
+ *   slot       0 or 1: which staging half (and which set of events) this step uses; alternate
+ *              them, and call zsm_decode_step_host_wait(slot) before reusing a slot's host
+ *              buffers.  At most one step per slot is in flight.
+ * The first call creates two streams and six events (no device memory) that live until
+ * zsm_cache_free; make it outside any stream capture.  wait: ZSM_ERR_STATE if the slot was
+ * never used. */
+zsm_status_t zsm_decode_host_layout(const zsm_cache_t *c, int32_t layer, size_t *q_off,
+                                    size_t *k_off, size_t *v_off, size_t *in_bytes,
+                                    size_t *out_bytes);
+zsm_status_t zsm_decode_step_host_async(zsm_cache_t *c, int32_t layer, const void *in_host,
+                                        void *out_host, void *staging, size_t staging_bytes,
+                                        int32_t slot, zsm_stream_t stream);
+zsm_status_t zsm_decode_step_host_wait(zsm_cache_t *c, int32_t slot);
+
 /* Decode attention over an UNCOMPRESSED cache [Eq. (att_score), Sec. 3.1]: what the paper's
  * FullKV baseline computes per step, for the cache path only -- the same-hardware comparator of
  * zsm_decode_step (Sec. 4.2 compares the two end to end).  No cache handle: the caller owns K and V.

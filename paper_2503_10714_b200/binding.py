@@ -43,7 +43,8 @@ SYMBOLS = ["zsm_split_budget", "zsm_cache_bytes", "zsm_cache_create", "zsm_cache
            "zsm_decode_step", "zsm_decode_staging_bytes", "zsm_decode_step_host",
            "zsm_unit_capacity", "zsm_cache_export_unit", "zsm_cache_import_unit",
            "zsm_last_device_status", "zsm_decode_launch_info", "zsm_status_string",
-           "zsm_selftest_wait_timeout"]
+           "zsm_selftest_wait_timeout", "zsm_decode_host_layout", "zsm_decode_step_host_async",
+           "zsm_decode_step_host_wait"]
 
 
 class ZsmConfig(C.Structure):
@@ -89,6 +90,9 @@ _lib.zsm_fullkv_decode.argtypes = [_i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, 
 _lib.zsm_fullkv_status.argtypes = [_vp, _vp]
 _lib.zsm_decode_staging_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
 _lib.zsm_decode_step_host.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.zsm_decode_host_layout.argtypes = [_vp, _i32] + [C.POINTER(_sz)] * 5
+_lib.zsm_decode_step_host_async.argtypes = [_vp, _i32, _vp, _vp, _vp, _sz, _i32, _vp]
+_lib.zsm_decode_step_host_wait.argtypes = [_vp, _i32]
 _lib.zsm_unit_capacity.argtypes = [_vp, _i32, _i32, _pi32, _pi32]
 _lib.zsm_cache_export_unit.argtypes = [_vp, _i32, _i32, _i32] + [_vp] * 8 + [_vp]
 _lib.zsm_cache_import_unit.argtypes = [_vp, _i32, _i32, _i32] + [_vp] * 8 + [_vp]
@@ -360,6 +364,35 @@ def zsm_decode_step_host(cache, layer, q_host, k_new_host, v_new_host, out_host,
     _check(_lib.zsm_decode_step_host(cache, layer, pq, pk, pv, po,
                                      _dev(staging, "staging", device=cache.device), _nbytes(staging),
                                      _stream(stream)), "zsm_decode_step_host")
+
+
+def zsm_decode_host_layout(cache, layer):
+    """(q_off, k_off, v_off, in_bytes, out_bytes) of the packed host input of the pipelined step."""
+    v = [_sz() for _ in range(5)]
+    _check(_lib.zsm_decode_host_layout(cache, _layer_arg(cache, layer, True), *[C.byref(x) for x in v]),
+           "zsm_decode_host_layout")
+    return tuple(x.value for x in v)
+
+
+def zsm_decode_step_host_async(cache, layer, in_host, out_host, staging, slot, stream=None):
+    """Enqueues one pipelined host-buffer step on staging half `slot` (0 or 1): in_host is a pinned
+    uint8 tensor laid out by zsm_decode_host_layout, out_host a pinned tensor of the cache's dtype."""
+    layer = _layer_arg(cache, layer, True)
+    _, _, _, in_bytes, out_bytes = zsm_decode_host_layout(cache, layer)
+    for name, t in (("in_host", in_host), ("out_host", out_host)):
+        if not isinstance(t, torch.Tensor) or t.is_cuda or not t.is_contiguous() or not t.is_pinned():
+            raise TypeError(f"{name}: a contiguous pinned host tensor is required")
+    if _nbytes(in_host) < in_bytes or _nbytes(out_host) < out_bytes:
+        raise ValueError("zsm_decode_step_host_async: host buffer smaller than zsm_decode_host_layout says")
+    _check(_lib.zsm_decode_step_host_async(cache, layer, C.c_void_p(in_host.data_ptr()),
+                                           C.c_void_p(out_host.data_ptr()),
+                                           _dev(staging, "staging", device=cache.device),
+                                           _nbytes(staging), int(slot), _stream(stream)),
+           "zsm_decode_step_host_async")
+
+
+def zsm_decode_step_host_wait(cache, slot):
+    _check(_lib.zsm_decode_step_host_wait(cache, int(slot)), "zsm_decode_step_host_wait")
 
 
 def zsm_unit_capacity(cache, layer, h):

@@ -70,6 +70,12 @@ struct zsm_cache {
     // only if that kernel is known not to write it: the last call on the same stream was this
     // library's and wrote a different single layer.  (Whatever else the caller put in between
     // was launched the ordinary way, after our call had completed.)
+    // Pipelined host-buffer steps (zsm_decode_step_host_async): two copy streams and three
+    // events per staging half, created on first use.
+    cudaStream_t cs_in = nullptr, cs_out = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_kernel[2] = {nullptr, nullptr},
+                ev_out[2] = {nullptr, nullptr};
+    bool slot_used[2] = {false, false};
     static constexpr int32_t kWroteAll = -1;
     std::unordered_map<cudaStream_t, int32_t> last_write;
     void wrote(cudaStream_t s, int32_t layer) {
@@ -425,7 +431,8 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
                 // Two CTAs of this shape fit on an SM when each stays within half of its shared
                 // memory (less the per-CTA reserve): the next layer's launch can then settle in
                 // beside this one's and have its first tiles in flight before this one ends.
-                // Taken when it leaves at least three ring stages; otherwise the whole SM.
+                // Taken when it leaves at least five ring stages (c5's grouped heads leave three:
+                // 25.5 us per layer against 23.9 with the whole SM); otherwise the whole SM.
                 // (Keeping the merged keys out of shared memory to gain a stage loses: the tail
                 // warp's reads of them are then the last thing the launch waits for; c4 14.9 ->
                 // 16.4 us per layer.)
@@ -434,7 +441,7 @@ zsm_status_t zsm_cache_create(const zsm_config_t *cfg, void *dev_buf, size_t byt
                 if (warps <= kPairConsumerWarps && (cfg->tune_stages == 0 || cfg->tune_stages <= 7)) {
                     st = fit_stages(pair_budget);
                     if (cfg->tune_stages > 0) st = std::min(st, (int)cfg->tune_stages);
-                    if (st < 3) st = 0;
+                    if (st < 5) st = 0;
                 }
                 if (st == 0) {
                     st = fit_stages(kMaxSmemPerCta);
@@ -518,6 +525,13 @@ zsm_status_t zsm_cache_reset(zsm_cache_t *c, zsm_stream_t stream) {
 
 zsm_status_t zsm_cache_free(zsm_cache_t *c) {
     if (!c) return ZSM_ERR_INVALID_ARG;
+    for (int s = 0; s < 2; ++s) {
+        if (c->ev_in[s]) cudaEventDestroy(c->ev_in[s]);
+        if (c->ev_kernel[s]) cudaEventDestroy(c->ev_kernel[s]);
+        if (c->ev_out[s]) cudaEventDestroy(c->ev_out[s]);
+    }
+    if (c->cs_in) cudaStreamDestroy(c->cs_in);
+    if (c->cs_out) cudaStreamDestroy(c->cs_out);
     delete c;
     return ZSM_OK;
 }
@@ -639,6 +653,68 @@ zsm_status_t zsm_decode_step_host(zsm_cache_t *c, int32_t layer, const void *q_h
     e = cudaMemcpyAsync(out_host, so, qn, cudaMemcpyDeviceToHost, cs);
     if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
     return cuda_status(e);
+}
+
+zsm_status_t zsm_decode_host_layout(const zsm_cache_t *c, int32_t layer, size_t *q_off,
+                                    size_t *k_off, size_t *v_off, size_t *in_bytes,
+                                    size_t *out_bytes) {
+    if (!c || layer < -1 || layer >= c->s.L) return ZSM_ERR_INVALID_ARG;
+    const size_t nu = layer < 0 ? c->s.n_units : c->s.upl;
+    const size_t qb = align_up(nu * c->s.G * c->s.row_bytes), kb = align_up(nu * c->s.row_bytes);
+    if (q_off) *q_off = 0;
+    if (k_off) *k_off = qb;
+    if (v_off) *v_off = qb + kb;
+    if (in_bytes) *in_bytes = qb + 2 * kb;
+    if (out_bytes) *out_bytes = nu * c->s.G * c->s.row_bytes;
+    return ZSM_OK;
+}
+
+zsm_status_t zsm_decode_step_host_async(zsm_cache_t *c, int32_t layer, const void *in_host,
+                                        void *out_host, void *staging, size_t staging_bytes,
+                                        int32_t slot, zsm_stream_t stream) {
+    if (!c || !in_host || !out_host || !staging || (slot != 0 && slot != 1))
+        return ZSM_ERR_INVALID_ARG;
+    size_t k_off = 0, v_off = 0, in_bytes = 0, out_bytes = 0;
+    zsm_status_t st = zsm_decode_host_layout(c, layer, nullptr, &k_off, &v_off, &in_bytes, &out_bytes);
+    if (st != ZSM_OK) return st;
+    const size_t half = in_bytes + align_up(out_bytes);
+    if (staging_bytes < 2 * half) return ZSM_ERR_BUFFER_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(staging) % kAlign != 0) return ZSM_ERR_INVALID_ARG;
+    if (!c->cs_in) {
+        bool ok = cudaStreamCreateWithFlags(&c->cs_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&c->cs_out, cudaStreamNonBlocking) == cudaSuccess;
+        for (int s = 0; s < 2 && ok; ++s)
+            ok = cudaEventCreateWithFlags(&c->ev_in[s], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_kernel[s], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_out[s], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return ZSM_ERR_CUDA;
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    uint8_t *sin = static_cast<uint8_t *>(staging) + (size_t)slot * half, *sout = sin + in_bytes;
+    cudaError_t e = cudaSuccess;
+    // copy in, once the kernel that last read this half has finished
+    if (c->slot_used[slot]) e = cudaStreamWaitEvent(c->cs_in, c->ev_kernel[slot], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sin, in_host, in_bytes, cudaMemcpyHostToDevice, c->cs_in);
+    if (e == cudaSuccess) e = cudaEventRecord(c->ev_in[slot], c->cs_in);
+    // the step, once its inputs are in and the previous result of this half has left
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_in[slot], 0);
+    if (e == cudaSuccess && c->slot_used[slot]) e = cudaStreamWaitEvent(cs, c->ev_out[slot], 0);
+    if (e != cudaSuccess) return ZSM_ERR_CUDA;
+    st = zsm_decode_step(c, layer, sin, sin + k_off, sin + v_off, sout, nullptr, nullptr, stream);
+    if (st != ZSM_OK) return st;
+    e = cudaEventRecord(c->ev_kernel[slot], cs);
+    // copy out
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->cs_out, c->ev_kernel[slot], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, sout, out_bytes, cudaMemcpyDeviceToHost, c->cs_out);
+    if (e == cudaSuccess) e = cudaEventRecord(c->ev_out[slot], c->cs_out);
+    c->slot_used[slot] = true;
+    return cuda_status(e);
+}
+
+zsm_status_t zsm_decode_step_host_wait(zsm_cache_t *c, int32_t slot) {
+    if (!c || (slot != 0 && slot != 1)) return ZSM_ERR_INVALID_ARG;
+    if (!c->slot_used[slot]) return ZSM_ERR_STATE;
+    return cuda_status(cudaEventSynchronize(c->ev_out[slot]));
 }
 
 zsm_status_t zsm_prefill_workspace_bytes(const zsm_cache_t *c, int32_t T, int32_t W,

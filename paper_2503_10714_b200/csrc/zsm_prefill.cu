@@ -15,6 +15,8 @@
 //   P5  prefill_gather     survivors' rows, scores and positions into the unit's slots
 #include "zsm_prefill.cuh"
 
+#include <algorithm>
+
 namespace zsm {
 
 namespace {
@@ -128,56 +130,81 @@ __global__ void __launch_bounds__(256) prefill_logits_kernel(const PrefillParams
 // ---------------------------------------------------------------------------
 // P1a on the tensor cores (16-bit storage): the window scoring is a dense
 // (G*W) x d x T contraction, 32 flop per K byte at G*W = 32 -- above what plain
-// FMAs can do at HBM speed.  Same grid and outputs as prefill_logits_kernel.
-// Warp w owns positions 16w .. 16w+15 of the chunk: their A fragments are read once
-// (mma.sync m16n8k16, contraction index permuted as in the decode kernel) and reused
-// for every block of eight query rows.  Scaled, masked logits go through a shared
-// tile, which gives coalesced row writes and the per-row (max, sum exp) of the chunk.
+// FMAs can do at HBM speed.  Same outputs as prefill_logits_kernel.
+// Persistent CTAs, grid (CTAs per unit, units): CTA x of a unit takes the unit's chunks
+// x, x + gridDim.x, ...  A producer warp streams the chunks' keys (contiguous in memory:
+// one bulk copy per chunk) through a ring of shared-memory stages, so a chunk's load runs
+// under the chunks before it; eight consumer warps take a chunk each time: warp w owns its
+// positions 16w .. 16w+15, whose A fragments are read once (mma.sync m16n8k16, contraction
+// index permuted as in the decode kernel) -- the stage is handed back at once -- and reused
+// for every block of eight query rows.  Scaled, masked logits go through a shared tile,
+// which gives coalesced row writes and the per-row (max, sum exp) of the chunk.  A window of
+// at most 32 query rows (the usual case) is loaded once per CTA, not once per chunk.
 // ---------------------------------------------------------------------------
+constexpr int kP1Stages = 2;  // two CTAs of two stages per SM: four chunks in flight
+constexpr int kP1Threads = 288;  // 8 consumer warps + the producer warp
+enum : int32_t { WP1_PRODUCER = 41, WP1_CHUNK = 42 };
+
 template <typename T, int D>
-__global__ void __launch_bounds__(256) prefill_logits_mma_kernel(const PrefillParams p) {
+__global__ void __launch_bounds__(kP1Threads) prefill_logits_mma_kernel(const PrefillParams p) {
     static_assert(sizeof(T) == 2, "16-bit storage");
     constexpr int CH = kPrefillChunk;  // 128 positions = 8 warps x 16 rows
     constexpr int ROWB = D * 2;
     constexpr int SEG = ROWB / 64;
     constexpr int LT = CH + 4;         // padded tile row (floats)
-    extern __shared__ __align__(16) uint8_t smb[];
-    uint8_t *Ks = smb;                                   // [CH][ROWB]   keys of the chunk
-    uint8_t *Qs = Ks + CH * ROWB;                        // [kQB][ROWB]  current block of queries
-    float *lt = reinterpret_cast<float *>(Qs + kQB * ROWB);  // [kQB][LT] logits of the block
+    constexpr int STAGE = CH * ROWB;
+    extern __shared__ __align__(128) uint8_t smb[];
+    uint8_t *Kring = smb;                                        // [stages][CH][ROWB]
+    uint8_t *Qs = Kring + kP1Stages * STAGE;                     // [kQB][ROWB] block of queries
+    float *lt = reinterpret_cast<float *>(Qs + kQB * ROWB);      // [kQB][LT] logits of the block
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(lt + kQB * LT);
+    uint64_t *empty_bar = full_bar + kP1Stages;
+    volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(empty_bar + kP1Stages);
 
     const int ul = blockIdx.y;
     const int b = ul / p.n_kv_heads, h = ul % p.n_kv_heads;
-    const int t0 = blockIdx.x * CH;
     const int T_len = p.T, W = p.W, G = p.G, GW = p.G * p.W;
-    const int n_chunks = gridDim.x;
+    const int n_chunks = (T_len + CH - 1) / CH;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tig = lane & 3;
     const uint8_t *Kg = static_cast<const uint8_t *>(p.K) + ((size_t)ul * T_len) * ROWB;
     const int n_q_heads = p.n_kv_heads * G;
 
-    for (int k = tid; k < CH * (ROWB / 16); k += 256) {
-        const int r = k / (ROWB / 16), c = k % (ROWB / 16);
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (t0 + r < T_len) v = *reinterpret_cast<const uint4 *>(Kg + (size_t)(t0 + r) * ROWB + c * 16);
-        *reinterpret_cast<uint4 *>(Ks + r * ROWB + c * 16) = v;
+    if (tid == 0) {
+        for (int s = 0; s < kP1Stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 8);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    // this warp's 16 positions as A fragments, all segments
-    uint4 fa[SEG], fc[SEG];
-    {
-        const uint8_t *pa = Ks + (warp * 16 + gq) * ROWB + tig * 16;
-#pragma unroll
-        for (int j = 0; j < SEG; ++j) {
-            fa[j] = *reinterpret_cast<const uint4 *>(pa + j * 64);
-            fc[j] = *reinterpret_cast<const uint4 *>(pa + 8 * ROWB + j * 64);
-        }
-    }
-    float *logits = reinterpret_cast<float *>(p.ws + p.wl.logits) + (size_t)ul * GW * T_len;
-    float2 *partial = reinterpret_cast<float2 *>(p.ws + p.wl.partial) + (size_t)ul * GW * n_chunks;
 
-    for (int qb = 0; qb < GW; qb += kQB) {
-        __syncthreads();  // the previous block's tile and queries are no longer read
+    if (warp == 8) {  // producer
+        if (lane != 0) return;
+        int s = 0;
+        uint32_t ph = 0;
+        for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+            if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, p.status, WP1_PRODUCER)) {
+                // copies in flight land in this CTA's memory: wait for them before leaving
+                const uint64_t t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+                return;
+            }
+            const uint32_t bytes = static_cast<uint32_t>(min(CH, T_len - c * CH)) * ROWB;
+            mbar_arrive_expect_tx(&full_bar[s], bytes);
+            bulk_g2s(Kring + (size_t)s * STAGE, Kg + (size_t)c * CH * ROWB, bytes, &full_bar[s]);
+            if (++s == kP1Stages) {
+                s = 0;
+                ph ^= 1u;
+            }
+        }
+        return;
+    }
+
+    auto csync = [&]() { named_bar_sync(1, 256); };
+    auto load_queries = [&](int qb) {
         for (int k = tid; k < kQB * (ROWB / 16); k += 256) {
             const int r = k / (ROWB / 16), c = k % (ROWB / 16);
             const int gw = qb + r;
@@ -189,58 +216,103 @@ __global__ void __launch_bounds__(256) prefill_logits_mma_kernel(const PrefillPa
             }
             *reinterpret_cast<uint4 *>(Qs + r * ROWB + c * 16) = v;
         }
-        __syncthreads();
-#pragma unroll
-        for (int nb = 0; nb < kQB / 8; ++nb) {
-            float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-            const uint8_t *pq = Qs + (nb * 8 + gq) * ROWB + tig * 16;
+    };
+    const bool one_block = GW <= kQB;  // the whole window fits the query block: load it once
+    if (one_block) {
+        load_queries(0);
+        csync();
+    }
+    float *logits = reinterpret_cast<float *>(p.ws + p.wl.logits) + (size_t)ul * GW * T_len;
+    float2 *partial = reinterpret_cast<float2 *>(p.ws + p.wl.partial) + (size_t)ul * GW * n_chunks;
+
+    int cs = 0;
+    uint32_t cph = 0;
+    for (int chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const int t0 = chunk * CH;
+        if (!mbar_wait_bounded(&full_bar[cs], cph, abort_flag, p.status, WP1_CHUNK)) return;
+        // this warp's 16 positions as A fragments, all segments (kept for every block of query
+        // rows); rows past the prompt's end hold leftovers of an earlier chunk: their logits are
+        // masked below, never summed
+        uint4 fa[SEG], fc[SEG];
+        {
+            const uint8_t *pa = Kring + (size_t)cs * STAGE + (warp * 16 + gq) * ROWB + tig * 16;
 #pragma unroll
             for (int j = 0; j < SEG; ++j) {
-                const uint4 qv = *reinterpret_cast<const uint4 *>(pq + j * 64);
-                mma_16x8x16<T>(c0, fa[j].x, fc[j].x, fa[j].y, fc[j].y, qv.x, qv.y);
-                mma_16x8x16<T>(c1, fa[j].z, fc[j].z, fa[j].w, fc[j].w, qv.z, qv.w);
+                fa[j] = *reinterpret_cast<const uint4 *>(pa + j * 64);
+                fc[j] = *reinterpret_cast<const uint4 *>(pa + 8 * ROWB + j * 64);
             }
-            // rows gq, gq+8 of the warp's positions; query rows nb*8 + tig*2, +1
-            const int pos = warp * 16 + gq;
-            const int qr = nb * 8 + tig * 2;
-            lt[qr * LT + pos] = (c0[0] + c1[0]) * p.scale;
-            lt[(qr + 1) * LT + pos] = (c0[1] + c1[1]) * p.scale;
-            lt[qr * LT + pos + 8] = (c0[2] + c1[2]) * p.scale;
-            lt[(qr + 1) * LT + pos + 8] = (c0[3] + c1[3]) * p.scale;
         }
-        __syncthreads();
-        // warp w: query rows 4w .. 4w+3 of the block; lane: positions lane + 32 i
-#pragma unroll
-        for (int jr = 0; jr < 4; ++jr) {
-            const int gw = qb + warp * 4 + jr;
-            if (gw >= GW) continue;  // uniform per warp
-            const int tau = T_len - W + (gw % W);  // the query's own position: keys 0..tau
-            float m = -INFINITY;
-            float lg[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int t = t0 + lane + 32 * i;
-                lg[i] = (t < T_len && t <= tau) ? lt[(warp * 4 + jr) * LT + lane + 32 * i] : -INFINITY;
-                if (t < T_len) logits[(size_t)gw * T_len + t] = lg[i];
-                m = fmaxf(m, lg[i]);
+        const int rel_stage = cs;
+        if (++cs == kP1Stages) {
+            cs = 0;
+            cph ^= 1u;
+        }
+        for (int qb = 0; qb < GW; qb += kQB) {
+            if (!one_block) {
+                csync();  // the previous block's tile and queries are no longer read
+                load_queries(qb);
             }
+            csync();      // queries in place; the previous chunk's tile is no longer read
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-            float sum = 0.f;
-            if (m > -INFINITY) {
+            for (int nb = 0; nb < kQB / 8; ++nb) {
+                float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint8_t *pq = Qs + (nb * 8 + gq) * ROWB + tig * 16;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sum += expf(lg[i] - m);
+                for (int j = 0; j < SEG; ++j) {
+                    const uint4 qv = *reinterpret_cast<const uint4 *>(pq + j * 64);
+                    mma_16x8x16<T>(c0, fa[j].x, fc[j].x, fa[j].y, fc[j].y, qv.x, qv.y);
+                    mma_16x8x16<T>(c1, fa[j].z, fc[j].z, fa[j].w, fc[j].w, qv.z, qv.w);
+                }
+                // rows gq, gq+8 of the warp's positions; query rows nb*8 + tig*2, +1
+                const int pos = warp * 16 + gq;
+                const int qr = nb * 8 + tig * 2;
+                lt[qr * LT + pos] = (c0[0] + c1[0]) * p.scale;
+                lt[(qr + 1) * LT + pos] = (c0[1] + c1[1]) * p.scale;
+                lt[qr * LT + pos + 8] = (c0[2] + c1[2]) * p.scale;
+                lt[(qr + 1) * LT + pos + 8] = (c0[3] + c1[3]) * p.scale;
             }
+            if (qb == 0) {
+                // The stage goes back once the fragments have been used, not merely requested:
+                // an arrival issued right behind the shared-memory loads can be seen by the
+                // producer before their data has been read (measured: wrong logits).
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[rel_stage]);
+            }
+            csync();
+            // warp w: query rows 4w .. 4w+3 of the block; lane: positions lane + 32 i
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-            if (lane == 0) partial[(size_t)gw * n_chunks + blockIdx.x] = make_float2(m, sum);
+            for (int jr = 0; jr < 4; ++jr) {
+                const int gw = qb + warp * 4 + jr;
+                if (gw >= GW) continue;  // uniform per warp
+                const int tau = T_len - W + (gw % W);  // the query's own position: keys 0..tau
+                float m = -INFINITY;
+                float lg[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int t = t0 + lane + 32 * i;
+                    lg[i] = (t < T_len && t <= tau) ? lt[(warp * 4 + jr) * LT + lane + 32 * i] : -INFINITY;
+                    if (t < T_len) logits[(size_t)gw * T_len + t] = lg[i];
+                    m = fmaxf(m, lg[i]);
+                }
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                float sum = 0.f;
+                if (m > -INFINITY) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) sum += expf(lg[i] - m);
+                }
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                if (lane == 0) partial[(size_t)gw * n_chunks + chunk] = make_float2(m, sum);
+            }
         }
     }
 }
 
 template <int D>
 size_t logits_mma_smem_bytes() {
-    return (size_t)(kPrefillChunk + kQB) * D * 2 + (size_t)kQB * (kPrefillChunk + 4) * 4;
+    return (size_t)(kP1Stages * kPrefillChunk + kQB) * D * 2 + (size_t)kQB * (kPrefillChunk + 4) * 4 +
+           (size_t)(2 * kP1Stages) * 8 + 64;
 }
 
 // P1b: one thread per (unit, query row): fold the chunk partials.
@@ -1245,7 +1317,12 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
     if (p.Qw) {
         const size_t sm = (size_t)(kPrefillChunk + kQB) * (D + 4) * 4;
         if constexpr (sizeof(T) == 2)
-            prefill_logits_mma_kernel<T, D><<<dim3(n_chunks, p.units), 256, logits_mma_smem_bytes<D>(), stream>>>(p);
+        {
+            // at most two CTAs per SM over the whole launch -- one wave -- each walking its share
+            // of a unit's chunks
+            const int per_unit = std::max(1, std::min(n_chunks, (2 * p.n_sm) / p.units));
+            prefill_logits_mma_kernel<T, D><<<dim3(per_unit, p.units), kP1Threads, logits_mma_smem_bytes<D>(), stream>>>(p);
+        }
         else
             prefill_logits_kernel<T, D><<<dim3(n_chunks, p.units), 256, sm, stream>>>(p);
         const int rows = p.units * p.G * p.W;

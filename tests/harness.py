@@ -199,7 +199,10 @@ def prefill_check(oracle, cache: GpuCache, layer, b, h, K, V, Qw, dbg, stats: Pa
         s_gpu = dbg["scores"][b, h].cpu().numpy().astype(np.float64)
         rel = np.abs(s_gpu - res.scores) / np.maximum(np.abs(res.scores.astype(np.float64)), 1e-30)
         stats.max_score_rel = max(stats.max_score_rel, float(rel.max()))
-        assert rel.max() <= SCORE_RTOL, f"{tag}: prompt score relative error {rel.max():.3e}"
+        bad = np.flatnonzero(rel > SCORE_RTOL)
+        assert bad.size == 0, (f"{tag}: prompt score relative error {rel.max():.3e} at {bad.size} positions, "
+                               f"first {bad[:6].tolist()}, last {bad[-3:].tolist()}, 128-position chunks "
+                               f"{sorted(set((bad // 128).tolist()))[:24]}")
     else:
         res = unit.prefill_compress(f64(K[b, h]), f64(V[b, h]), scores=scores_given, **kw)
     r = res.report

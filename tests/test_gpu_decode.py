@@ -176,6 +176,51 @@ def test_host_buffer_entry_point_matches_device_entry_point(zb):
         a.close(), b.close()
 
 
+def test_pipelined_host_buffer_steps_match_device_entry_point(zb):
+    """zsm_decode_step_host_async over two staging halves: same outputs, step for step, as the
+    device entry point, with two steps in flight at a time."""
+    w = wl.Workload("hostpipe", 2, 2, 4, 2, 128, "bf16", 0, 0, 0, None, 39)
+    mk = lambda: GpuCache(zb, w, np.full((2, 2), 8), np.full((2, 2), 9), np.full((2, 2), 2))
+    a, b = mk(), mk()
+    try:
+        q_off, k_off, v_off, in_bytes, out_bytes = zb.zsm_decode_host_layout(b.h, -1)
+        half = in_bytes + (out_bytes + 255) // 256 * 256
+        staging = torch.empty(2 * half, dtype=torch.uint8, device="cuda")
+        ins = [torch.zeros(in_bytes, dtype=torch.uint8).pin_memory() for _ in range(2)]
+        outs = [torch.empty(w.n_layers, w.batch, w.n_q_heads, w.head_dim,
+                            dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_decode_step_host_wait(b.h, 0)
+        assert e.value.status == zb.ZSM_ERR_STATE
+        steps, ref = 41, []
+        for step in range(steps):
+            q, k, v = wl.decode_inputs(w, step)
+            out, _, _ = a.decode(q.cuda(), k.cuda(), v.cuda())
+            ref.append(out.cpu().clone())
+        def pack(dst, q, k, v):
+            for off, t in ((q_off, q), (k_off, k), (v_off, v)):
+                raw = t.contiguous().view(torch.uint8).reshape(-1)
+                dst[off:off + raw.numel()] = raw
+        got = [None] * steps
+        for step in range(steps + 1):
+            slot = step & 1
+            if step >= 2 or step == steps:
+                pass
+            if step >= 2:                       # the slot's previous step must be done before reuse
+                zb.zsm_decode_step_host_wait(b.h, slot)
+                got[step - 2] = outs[slot].clone()
+            if step < steps:
+                pack(ins[slot], *wl.decode_inputs(w, step))
+                zb.zsm_decode_step_host_async(b.h, -1, ins[slot], outs[slot], staging, slot)
+        zb.zsm_decode_step_host_wait(b.h, (steps - 1) & 1)
+        got[steps - 1] = outs[(steps - 1) & 1].clone()
+        for step in range(steps):
+            assert torch.equal(got[step], ref[step]), f"step {step}"
+        assert a.status() == 0 and b.status() == 0
+    finally:
+        a.close(), b.close()
+
+
 def test_runs_are_bitwise_reproducible(zb):
     w = wl.Workload("repro", 2, 2, 8, 2, 128, "bf16", 0, 0, 0, None, 17)
     outs = []

@@ -108,6 +108,43 @@ def test_layer_with_more_units_than_resident_ctas(zb, oracle):
         cache.close()
 
 
+def test_layers_compressed_side_by_side_on_two_streams(zb, oracle):
+    """Layers are independent: their prompt passes may run at the same time on different
+    streams, each with a workspace of its own.  Three layers on two streams (the third queues
+    behind the first), every unit of every layer checked against the oracle."""
+    w = wl.Workload("side", 3, 2, 4, 2, 128, "f16", 1800, 0, 16, None, 40)
+    bp, bc, br = np.full((3, 2), 24), np.full((3, 2), 40), np.array([[3, 40], [9, 5], [70, 2]])
+    cache = GpuCache(zb, w, bp, bc, br)
+    stats = ParityStats()
+    try:
+        streams = [torch.cuda.Stream() for _ in range(2)]
+        need = zb.zsm_prefill_workspace_bytes(cache.h, w.prompt_len, w.window)
+        wss = [torch.empty(need, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        prompts = [wl.prompt(w, layer) for layer in range(w.n_layers)]
+        dev = [[t.cuda() for t in pr] for pr in prompts]
+        dbgs = []
+        torch.cuda.synchronize()
+        for layer in range(w.n_layers):
+            T = w.prompt_len
+            d = {"scores": torch.empty(w.batch, w.n_kv_heads, T, dtype=torch.float32, device="cuda"),
+                 "evicted": torch.zeros(w.batch, w.n_kv_heads, T, dtype=torch.uint8, device="cuda"),
+                 "targets": torch.full((w.batch, w.n_kv_heads, T), -9, dtype=torch.int32, device="cuda")}
+            K, V, Qw = dev[layer]
+            zb.zsm_prefill_compress(cache.h, layer, K, V, Qw, None, T, w.window, wss[layer % 2],
+                                    d["scores"], d["evicted"], d["targets"], stream=streams[layer % 2])
+            dbgs.append(d)
+        torch.cuda.synchronize()
+        for layer in range(w.n_layers):
+            K, V, Qw = prompts[layer]
+            for b in range(w.batch):
+                for h in range(w.n_kv_heads):
+                    prefill_check(oracle, cache, layer, b, h, K, V, Qw, dbgs[layer], stats,
+                                  tag=f"side by side, unit {(layer, b, h)}")
+        assert cache.status() == 0 and stats.merges > 15000
+    finally:
+        cache.close()
+
+
 def test_supplied_scores_with_exact_ties(zb, oracle):
     """Scores given by the caller, drawn from four values only: the selection is decided by
     the position rule almost everywhere and must match the oracle bit for bit (no near tie
