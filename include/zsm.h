@@ -145,6 +145,9 @@ zsm_status_t zsm_prefill_workspace_bytes(const zsm_cache_t *c, int32_t T, int32_
  *            for query position tau), averaged over a group.  NULL to use `scores`.
  *   scores   dev fp32 [batch][n_kv_heads][T], used iff Qw is NULL
  *   workspace dev, >= zsm_prefill_workspace_bytes, 256-byte aligned
+ * Layers are independent: calls for different layers may run at the same time on different
+ * streams, each with a workspace of its own (the sequential merge chain of one layer keeps
+ * only one CTA per unit busy, so several layers in flight use the machine far better).
  * Optional dev outputs for inspection (NULL to skip), each [batch][n_kv_heads][T]:
  *   dbg_scores  fp32 score of every prompt position
  *   dbg_evicted uint8, 1 where the position was evicted (merged or dropped)
