@@ -213,6 +213,24 @@ zsm_status_t zsm_prefill_scores_full(zsm_cache_t *c, const void *K, const void *
                                      void *workspace, size_t workspace_bytes,
                                      zsm_stream_t stream);
 
+/* Causal prefill attention of one layer's prompt with the compression's inputs as by-products
+ * [Eq. (att_score) for every prompt query; App. B: the scores come from the prefill's attention
+ * history]: out[b][hq][tau] = sum_{t <= tau} a^(tau)_t v_t, the rows' log-sum-exp, and -- when
+ * `scores` is given -- the full-history scores of zsm_prefill_scores_full, ready for
+ * zsm_prefill_compress(scores = ...).  A model that runs this as its prefill attention needs no
+ * separate scoring pass.  Tensor cores throughout (tcgen05): row statistics, then the output as
+ * two products per key tile (Q K^T; weights exp(logit - lse) as 16-bit values times V), then the
+ * decayed column sums.
+ *   K, V    dev [batch][n_kv_heads][T][head_dim];  Q dev [batch][n_q_heads][T][head_dim];
+ *           storage dtype of the cache (fp16 or bf16; ZSM_ERR_UNSUPPORTED for fp32), 16-byte aligned
+ *   out     dev [batch][n_q_heads][T][head_dim], storage dtype, written
+ *   lse     dev fp32 [batch][n_q_heads][T], written (natural log of each row's sum of exponentials)
+ *   scores  dev fp32 [batch][n_kv_heads][T], written, or NULL
+ * Asynchronous on `stream`; nothing is allocated. */
+zsm_status_t zsm_prefill_attention(zsm_cache_t *c, const void *K, const void *V, const void *Q,
+                                   int32_t T, void *out, float *lse, float *scores,
+                                   zsm_stream_t stream);
+
 /* One decode step [Algorithm 1 with Eq. (att_score2)], one kernel launch.
  *   layer      0..n_layers-1: that layer's units; tensors have no layer dimension.
  *              -1: every layer in one launch; tensors carry a leading

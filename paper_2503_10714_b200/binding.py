@@ -44,7 +44,7 @@ SYMBOLS = ["zsm_split_budget", "zsm_cache_bytes", "zsm_cache_create", "zsm_cache
            "zsm_unit_capacity", "zsm_cache_export_unit", "zsm_cache_import_unit",
            "zsm_last_device_status", "zsm_decode_launch_info", "zsm_status_string",
            "zsm_selftest_wait_timeout", "zsm_decode_host_layout", "zsm_decode_step_host_async",
-           "zsm_decode_step_host_wait"]
+           "zsm_decode_step_host_wait", "zsm_prefill_attention"]
 
 
 class ZsmConfig(C.Structure):
@@ -83,6 +83,7 @@ _lib.zsm_prefill_compress_static.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _i32
                                              _vp, _vp]
 _lib.zsm_prefill_scores_full_workspace_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
 _lib.zsm_prefill_scores_full.argtypes = [_vp, _vp, _vp, _vp, _i32, _vp, _vp, _sz, _vp]
+_lib.zsm_prefill_attention.argtypes = [_vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
 _lib.zsm_decode_step.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.zsm_fullkv_workspace_bytes.argtypes = [_i32, _i32, _i32, _i32, C.POINTER(_sz)]
 _lib.zsm_fullkv_decode.argtypes = [_i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, C.c_float, _vp,
@@ -301,6 +302,19 @@ def zsm_prefill_scores_full(cache, K, Q, T, scores, workspace=None, lse=None, st
         _dev(scores, "scores", torch.float32, cache.batch * cache.n_kv_heads * T, dev),
         _dev(workspace, "workspace", device=dev), _nbytes(workspace), _stream(stream)),
         "zsm_prefill_scores_full")
+
+
+def zsm_prefill_attention(cache, K, V, Q, T, out, lse, scores=None, stream=None):
+    """Causal prefill attention of a prompt: writes `out` [batch][n_q_heads][T][d] (cache dtype),
+    `lse` fp32 [batch][n_q_heads][T] and, if given, the full-history `scores`
+    fp32 [batch][n_kv_heads][T]."""
+    T = int(T)
+    dt, dev, d = cache.torch_dtype, cache.device, cache.head_dim
+    nk, nq = cache.batch * cache.n_kv_heads * T, cache.batch * cache.n_q_heads * T
+    _check(_lib.zsm_prefill_attention(
+        cache, _dev(K, "K", dt, nk * d, dev), _dev(V, "V", dt, nk * d, dev), _dev(Q, "Q", dt, nq * d, dev), T,
+        _dev(out, "out", dt, nq * d, dev), _dev(lse, "lse", torch.float32, nq, dev),
+        _dev(scores, "scores", torch.float32, nk, dev), _stream(stream)), "zsm_prefill_attention")
 
 
 def _decode_args(cache: Cache, layer, q, k_new, v_new, out, host: bool):

@@ -808,6 +808,40 @@ zsm_status_t zsm_prefill_scores_full(zsm_cache_t *c, const void *K, const void *
     return rc == 0 ? ZSM_OK : ZSM_ERR_CUDA;
 }
 
+zsm_status_t zsm_prefill_attention(zsm_cache_t *c, const void *K, const void *V, const void *Q,
+                                   int32_t T, void *out, float *lse, float *scores,
+                                   zsm_stream_t stream) {
+    if (!c || !K || !V || !Q || !out || !lse || T < 1) return ZSM_ERR_INVALID_ARG;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(Q) || !aligned16(out)) return ZSM_ERR_INVALID_ARG;
+    if (c->s.dtype == ZSM_F32) return ZSM_ERR_UNSUPPORTED;
+    if ((long)c->s.B * c->s.Hq > 65535) return ZSM_ERR_UNSUPPORTED;
+    FullScoreParams p;
+    p.K = K;
+    p.Q = Q;
+    p.status = reinterpret_cast<int32_t *>(c->base + c->lay.status);
+    p.batch = c->s.B;
+    p.n_kv_heads = c->s.Hkv;
+    p.G = c->s.G;
+    p.T = T;
+    p.lambda = c->lambda;
+    p.scale = c->scale;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    // row statistics first (and, when asked for, the decayed column sums from them) ...
+    p.lse = nullptr;
+    p.lse_out = lse;
+    p.scores = scores;
+    int rc = scores ? launch_full_scores(c->s.dtype, c->s.D, p, cs)
+                    : launch_row_statistics(c->s.dtype, c->s.D, p, cs);
+    if (rc == -1) return ZSM_ERR_UNSUPPORTED;
+    if (rc != 0) return ZSM_ERR_CUDA;
+    // ... then the output, whose weights exp(logit - lse) need no running maximum
+    p.lse = lse;
+    p.lse_out = nullptr;
+    rc = launch_attention_output(c->s.dtype, c->s.D, p, V, out, cs);
+    if (rc == -1) return ZSM_ERR_UNSUPPORTED;
+    return rc == 0 ? ZSM_OK : ZSM_ERR_CUDA;
+}
+
 zsm_status_t zsm_cache_export_unit(zsm_cache_t *c, int32_t layer, int32_t b, int32_t h,
                                    float *K, float *V, float *score, int32_t *pos, float *Kr,
                                    float *Vr, uint32_t *w, int32_t *counters,

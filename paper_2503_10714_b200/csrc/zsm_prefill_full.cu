@@ -437,6 +437,284 @@ __global__ void __launch_bounds__(kTcThreads, 2)
                      : "memory");
 }
 
+// ---------------------------------------------------------------------------
+// Causal attention output of the prompt, o_tau = sum_{t <= tau} a^(tau)_t v_t [Eq. (att_score)], from
+// the rows' log-sum-exp of pass 1: with the normaliser known no running maximum is needed, so a
+// tile's weights exp(logit - lse) are final when they are computed.  Per CTA a block of 128
+// queries of one head is resident; for every key tile up to the diagonal
+//   product 1   S = Q K^T            (tcgen05.mma, two accumulators of 128 columns, as above)
+//   epilogue    P = exp2(S * scale - lse) as 16-bit values, written to shared memory in the
+//               K-major 128-byte-swizzled layout the tensor map gives an operand tile
+//   product 2   O += P V             (tcgen05.mma; V's tile, rows = keys, is the N x K operand in
+//               "MN-major" form: N = head dimension contiguous)
+// O is a third accumulator (128 lanes x d columns), read back once at the end.  One warp requests
+// tiles and issues both products, eight warps do the exponentials.  384 (320) tensor-memory
+// columns: one CTA per SM.
+// ---------------------------------------------------------------------------
+constexpr int kAoThreads = kTcEpiThreads + 32;
+enum : int32_t { WA_S = 51, WA_P = 52, WA_PFREE = 53, WA_K = 54, WA_V = 55, WA_VFREE = 56, WA_SFREE = 57, WA_O = 58, WA_Q = 59 };
+
+template <int D>
+struct AoSmem {
+    static constexpr int KB = D / kTcKBlock;
+    static constexpr int KBLOCK = kTcRows * 128;
+    static constexpr int TILE = KB * KBLOCK;          // Q, K or V tile
+    static constexpr int PTILE = 2 * KBLOCK;          // 128 queries x 128 keys, 16 bit
+    static constexpr int q = 0;
+    static constexpr int k = TILE;                    // two stages
+    static constexpr int v = k + 2 * TILE;            // two stages
+    static constexpr int pw = v + 2 * TILE;           // the weights of the tile in hand
+    static constexpr int bars = pw + 2 * PTILE;       // high parts, then (bf16 only) the remainders
+    static constexpr int total = bars + 256 + 1024;   // + slack to align the base to 1 KiB
+    static constexpr int tmem_cols = 512;             // 2 x 128 (S) + D (O), rounded up to a power of two
+};
+
+// V tile as the N x K operand with N (head dimension) contiguous: 64 elements per 128-byte row,
+// 8 keys per swizzle atom; the other 64 elements of d one block on (leading offset), the next 8
+// keys 1024 bytes on (stride offset).  `kstep`: 16 keys = two atoms.
+template <int D>
+__device__ __forceinline__ uint64_t umma_desc_v_mn(const uint8_t *tile, int kstep) {
+    const uint64_t a = ((smem_u32(tile) + static_cast<uint32_t>(kstep) * 2048u) >> 4) & 0x3fffu;
+    return a | (static_cast<uint64_t>(AoSmem<D>::KBLOCK >> 4) << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kAoThreads, 1)
+    attn_out_tc_kernel(const FullScoreParams p, void *out_ptr, const __grid_constant__ CUtensorMap map_k,
+                       const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_q) {
+    using L = AoSmem<D>;
+    using E = Elem<T>;
+    constexpr int KS = D / 16;
+    // bf16 keeps 8 bits of a weight: it is written as a high part and a remainder (two products
+    // per step), which brings the weights to 16 bits; fp16's 11 bits are enough for a 16-bit output
+    constexpr bool kSplitW = E::kIsBf16;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t *q_bar = reinterpret_cast<uint64_t *>(smem + L::bars);
+    uint64_t *k_full = q_bar + 1;      // [2] key tile landed
+    uint64_t *v_full = k_full + 2;     // [2] value tile landed
+    uint64_t *v_free = v_full + 2;     // [2] product 2 done with the value tile (and with the weights)
+    uint64_t *s_ready = v_free + 2;    // [2] product 1 complete
+    uint64_t *s_free = s_ready + 2;    // [2] accumulator read by the eight warps
+    uint64_t *p_ready = s_free + 2;    // weights written by the eight warps
+    uint64_t *p_free = p_ready + 1;    // product 2 has read the weights
+    uint64_t *o_done = p_free + 1;     // every product complete
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(o_done + 1);
+    volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(tmem_slot + 2);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Tn = p.T, G = p.G;
+    const int nb = (Tn + kTcRows - 1) / kTcRows;
+    const int rb = nb - 1 - blockIdx.x;  // the longest blocks first
+    const int b = blockIdx.y / (p.n_kv_heads * G);
+    const int hq = blockIdx.y % (p.n_kv_heads * G);
+    const int zk = b * p.n_kv_heads + hq / G;
+    const int zq = b * p.n_kv_heads * G + hq;
+    const int n_tiles = rb + 1;
+    const float scale2 = p.scale * kLog2e;
+
+    if (tid == 0) {
+        mbar_init(q_bar, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&k_full[s], 1);
+            mbar_init(&v_full[s], 1);
+            mbar_init(&v_free[s], 1);
+            mbar_init(&s_ready[s], 1);
+            mbar_init(&s_free[s], kTcEpiThreads / 32);
+        }
+        mbar_init(p_ready, kTcEpiThreads / 32);
+        mbar_init(p_free, 1);
+        mbar_init(o_done, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(tmem_slot)),
+                     "r"(L::tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base + 2 * kTcRows;
+
+    const uint32_t f = E::kIsBf16 ? 1u : 0u;
+    const uint32_t idesc_s = (1u << 4) | (f << 7) | (f << 10) | ((kTcRows >> 3) << 17) | ((kTcRows >> 4) << 24);
+    // product 2: B (the value tile) is "MN-major" (bit 16), N = D
+    const uint32_t idesc_o = (1u << 4) | (f << 7) | (f << 10) | (1u << 16) | ((static_cast<uint32_t>(D) >> 3) << 17) |
+                             ((kTcRows >> 4) << 24);
+    bool ok = true;
+    const bool producer = warp == kTcEpiThreads / 32;
+
+    if (producer) {
+        if (lane == 0) {
+            auto load_tile = [&](uint8_t *dst, const CUtensorMap *map, int z, int jb, uint64_t *bar) {
+                mbar_arrive_expect_tx(bar, L::TILE);
+#pragma unroll
+                for (int kb = 0; kb < L::KB; ++kb)
+                    tma_load_3d(dst + kb * L::KBLOCK, map, kb * kTcKBlock, jb * kTcRows, z, bar);
+            };
+            load_tile(smem + L::q, &map_q, zq, rb, q_bar);
+            for (int i = 0; i < 2 && i < n_tiles; ++i) {
+                load_tile(smem + L::k + i * L::TILE, &map_k, zk, i, &k_full[i]);
+                load_tile(smem + L::v + i * L::TILE, &map_v, zk, i, &v_full[i]);
+            }
+            // product 2 of tile t: needs its weights and its value tile
+            auto issue_pv = [&](int t) {
+                if (!mbar_wait_bounded(p_ready, t & 1u, abort_flag, p.status, WA_P)) return false;
+                // the weights exist, so product 1 of tile t is complete: its key stage is free
+                if (t + 2 < n_tiles)
+                    load_tile(smem + L::k + (t & 1) * L::TILE, &map_k, zk, t + 2, &k_full[t & 1]);
+                if (!mbar_wait_bounded(&v_full[t & 1], (t >> 1) & 1u, abort_flag, p.status, WA_V)) return false;
+                tc_fence_after();
+                const uint8_t *vt = smem + L::v + (t & 1) * L::TILE;
+#pragma unroll
+                for (int ks = 0; ks < kTcRows / 16; ++ks) {
+                    const int o = (ks / 4) * L::KBLOCK + (ks % 4) * 32;  // 16 keys = 32 bytes of a weight row
+                    umma_f16_ss(tmem_o, umma_desc_sw128(smem + L::pw + o), umma_desc_v_mn<D>(vt, ks), idesc_o,
+                                (t > 0 || ks > 0) ? 1u : 0u);
+                    if constexpr (kSplitW)
+                        umma_f16_ss(tmem_o, umma_desc_sw128(smem + L::pw + L::PTILE + o), umma_desc_v_mn<D>(vt, ks),
+                                    idesc_o, 1u);
+                }
+                umma_commit(p_free);
+                umma_commit(&v_free[t & 1]);
+                return true;
+            };
+            ok = mbar_wait_bounded(q_bar, 0, abort_flag, p.status, WA_Q);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                ok = mbar_wait_bounded(&k_full[j & 1], (j >> 1) & 1u, abort_flag, p.status, WA_K);
+                if (ok && j >= 2)
+                    ok = mbar_wait_bounded(&s_free[j & 1], ((j - 2) >> 1) & 1u, abort_flag, p.status, WA_SFREE);
+                if (!ok) break;
+                tc_fence_after();
+                const uint8_t *kt = smem + L::k + (j & 1) * L::TILE;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int o = (ks / 4) * L::KBLOCK + (ks % 4) * 32;
+                    umma_f16_ss(tmem_base + (j & 1) * kTcRows, umma_desc_sw128(smem + L::q + o),
+                                umma_desc_sw128(kt + o), idesc_s, ks > 0);
+                }
+                umma_commit(&s_ready[j & 1]);
+                if (j >= 1) ok = issue_pv(j - 1);
+                if (ok && j >= 2) {
+                    // value stage of tile j - 2 (the one tile j will use) is free once its product is done
+                    ok = mbar_wait_bounded(&v_free[j & 1], ((j - 2) >> 1) & 1u, abort_flag, p.status, WA_VFREE);
+                    if (ok) load_tile(smem + L::v + (j & 1) * L::TILE, &map_v, zk, j, &v_full[j & 1]);
+                }
+            }
+            if (ok) ok = issue_pv(n_tiles - 1);
+            if (ok) umma_commit(o_done);
+            if (!ok) {
+                const uint64_t t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    } else {
+        // eight warps: accumulator lanes 32 quad .., columns 64 cq ..
+        const int quad = warp & 3, cq = warp >> 2;
+        const int rloc = quad * 32 + lane;
+        const int row = rb * kTcRows + rloc;
+        const float lse2 = row < Tn ? p.lse[(size_t)zq * Tn + row] * kLog2e : 0.f;
+        uint8_t *prow = smem + L::pw + cq * L::KBLOCK + rloc * 128;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait_bounded(&s_ready[buf], (j >> 1) & 1u, abort_flag, p.status, WA_S)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const bool diag = j == rb;
+            uint32_t w[32];  // 64 weights of this thread's row, packed in pairs
+            uint32_t wl[kSplitW ? 32 : 1];  // their remainders
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kTcRows + cq * 64 + c * 32, v);
+                if (c == 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s_free[buf]);
+                }
+                const int col0 = j * kTcRows + cq * 64 + c * 32;
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float x0 = ex2(fmaf(__uint_as_float(v[e]), scale2, -lse2));
+                    float x1 = ex2(fmaf(__uint_as_float(v[e + 1]), scale2, -lse2));
+                    if (row >= Tn || (diag && col0 + e > row)) x0 = 0.f;       // keep key <= query
+                    if (row >= Tn || (diag && col0 + e + 1 > row)) x1 = 0.f;
+                    if constexpr (E::kIsBf16) {
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                        const float2 hb = __bfloat1622float2(h);
+                        const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - hb.x, x1 - hb.y);
+                        w[c * 16 + e / 2] = *reinterpret_cast<const uint32_t *>(&h);
+                        wl[c * 16 + e / 2] = *reinterpret_cast<const uint32_t *>(&l);
+                    } else {
+                        const __half2 h = __floats2half2_rn(x0, x1);
+                        w[c * 16 + e / 2] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                }
+            }
+            // the weights of the tile before this one have been multiplied
+            if (j >= 1 && !mbar_wait_bounded(p_free, (j - 1) & 1u, abort_flag, p.status, WA_PFREE)) {
+                ok = false;
+                break;
+            }
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch)  // 16-byte chunk ch of the row sits at chunk ch ^ (row % 8)
+            {
+                *reinterpret_cast<uint4 *>(prow + ((ch ^ (rloc & 7)) << 4)) =
+                    make_uint4(w[4 * ch], w[4 * ch + 1], w[4 * ch + 2], w[4 * ch + 3]);
+                if constexpr (kSplitW)
+                    *reinterpret_cast<uint4 *>(prow + L::PTILE + ((ch ^ (rloc & 7)) << 4)) =
+                        make_uint4(wl[4 * ch], wl[4 * ch + 1], wl[4 * ch + 2], wl[4 * ch + 3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_ready);
+        }
+        if (ok && mbar_wait_bounded(o_done, 0, abort_flag, p.status, WA_O)) {
+            tc_fence_after();
+            T *orow = static_cast<T *>(out_ptr) + ((size_t)zq * Tn + row) * D;
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c) {
+                // the eight warps split the d columns: half cq takes columns cq * D/2 ..
+                uint32_t v[32];
+                const int col = cq * (D / 2) + c * 32;
+                tmem_ld32(tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + col, v);
+                if (row < Tn) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float a0 = __uint_as_float(v[e + 2 * k]), a1 = __uint_as_float(v[e + 2 * k + 1]);
+                            if constexpr (E::kIsBf16) {
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
+                                pk[k] = *reinterpret_cast<const uint32_t *>(&h);
+                            } else {
+                                const __half2 h = __floats2half2_rn(a0, a1);
+                                pk[k] = *reinterpret_cast<const uint32_t *>(&h);
+                            }
+                        }
+                        *reinterpret_cast<uint4 *>(orow + col + e) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(L::tmem_cols)
+                     : "memory");
+}
+
 // cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link
 // against the driver library directly.
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -502,7 +780,56 @@ int prepare_full_one() {
     return static_cast<int>(e);
 }
 
+// Pass 1 alone: every query row's log-sum-exp into p.lse_out.
+template <typename T, int D>
+int launch_rows_one(const FullScoreParams &p, cudaStream_t stream) {
+    CUtensorMap map_k, map_q;
+    if (!make_map(&map_k, p.K, p.batch * p.n_kv_heads, p.T, D, Elem<T>::kIsBf16) ||
+        !make_map(&map_q, p.Q, p.batch * p.n_kv_heads * p.G, p.T, D, Elem<T>::kIsBf16))
+        return static_cast<int>(cudaErrorInvalidValue);
+    const int nres = (p.T + kTcRows - 1) / kTcRows;
+    const dim3 grid(nres, p.batch * p.n_kv_heads * p.G);
+    full_pass_tc_kernel<T, D, false><<<grid, kTcThreads, TcSmem<D>::total, stream>>>(p, map_k, map_q);
+    return static_cast<int>(cudaGetLastError());
+}
+
+template <typename T, int D>
+int launch_attn_one(const FullScoreParams &p, const void *V, void *out, cudaStream_t stream) {
+    CUtensorMap map_k, map_v, map_q;
+    if (!make_map(&map_k, p.K, p.batch * p.n_kv_heads, p.T, D, Elem<T>::kIsBf16) ||
+        !make_map(&map_v, V, p.batch * p.n_kv_heads, p.T, D, Elem<T>::kIsBf16) ||
+        !make_map(&map_q, p.Q, p.batch * p.n_kv_heads * p.G, p.T, D, Elem<T>::kIsBf16))
+        return static_cast<int>(cudaErrorInvalidValue);
+    const int nres = (p.T + kTcRows - 1) / kTcRows;
+    const dim3 grid(nres, p.batch * p.n_kv_heads * p.G);
+    attn_out_tc_kernel<T, D><<<grid, kAoThreads, AoSmem<D>::total, stream>>>(p, out, map_k, map_v, map_q);
+    return static_cast<int>(cudaGetLastError());
+}
+
+template <typename T, int D>
+int prepare_attn_one() {
+    return static_cast<int>(cudaFuncSetAttribute(attn_out_tc_kernel<T, D>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, AoSmem<D>::total));
+}
+
 }  // namespace
+
+int launch_attention_output(int dtype, int D, const FullScoreParams &p, const void *V, void *out,
+                            cudaStream_t stream) {
+    if (dtype == 1 && D == 64) return launch_attn_one<__half, 64>(p, V, out, stream);
+    if (dtype == 1 && D == 128) return launch_attn_one<__half, 128>(p, V, out, stream);
+    if (dtype == 2 && D == 64) return launch_attn_one<__nv_bfloat16, 64>(p, V, out, stream);
+    if (dtype == 2 && D == 128) return launch_attn_one<__nv_bfloat16, 128>(p, V, out, stream);
+    return -1;
+}
+
+int launch_row_statistics(int dtype, int D, const FullScoreParams &p, cudaStream_t stream) {
+    if (dtype == 1 && D == 64) return launch_rows_one<__half, 64>(p, stream);
+    if (dtype == 1 && D == 128) return launch_rows_one<__half, 128>(p, stream);
+    if (dtype == 2 && D == 64) return launch_rows_one<__nv_bfloat16, 64>(p, stream);
+    if (dtype == 2 && D == 128) return launch_rows_one<__nv_bfloat16, 128>(p, stream);
+    return -1;
+}
 
 int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t stream) {
     if (dtype == 1 && D == 64) return launch_full_one<__half, 64>(p, stream);
@@ -513,11 +840,12 @@ int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t 
 }
 
 int prepare_full_scores(int dtype, int D) {
-    if (dtype == 1 && D == 64) return prepare_full_one<__half, 64>();
-    if (dtype == 1 && D == 128) return prepare_full_one<__half, 128>();
-    if (dtype == 2 && D == 64) return prepare_full_one<__nv_bfloat16, 64>();
-    if (dtype == 2 && D == 128) return prepare_full_one<__nv_bfloat16, 128>();
-    return -1;
+    int rc = -1;
+    if (dtype == 1 && D == 64) rc = prepare_full_one<__half, 64>() | prepare_attn_one<__half, 64>();
+    if (dtype == 1 && D == 128) rc = prepare_full_one<__half, 128>() | prepare_attn_one<__half, 128>();
+    if (dtype == 2 && D == 64) rc = prepare_full_one<__nv_bfloat16, 64>() | prepare_attn_one<__nv_bfloat16, 64>();
+    if (dtype == 2 && D == 128) rc = prepare_full_one<__nv_bfloat16, 128>() | prepare_attn_one<__nv_bfloat16, 128>();
+    return rc;
 }
 
 }  // namespace zsm

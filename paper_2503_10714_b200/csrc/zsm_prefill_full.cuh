@@ -21,6 +21,12 @@ struct FullScoreParams {
 // Enqueues one or both passes on `stream`: row statistics (skipped when p.lse is set), then the
 // decayed column sums.  dtype: 1 fp16, 2 bf16.  Returns a cudaError_t as int; -1: no kernel.
 int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t stream);
+// The first pass alone: every query row's log-sum-exp into p.lse_out.
+int launch_row_statistics(int dtype, int D, const FullScoreParams &p, cudaStream_t stream);
+// Causal attention output of the prompt from the rows' log-sum-exp (p.lse, required):
+// out [batch][n_q_heads][T][d] in the storage dtype; V [batch][n_kv_heads][T][d].
+int launch_attention_output(int dtype, int D, const FullScoreParams &p, const void *V, void *out,
+                            cudaStream_t stream);
 // Raises the kernels' dynamic shared-memory limit; returns a cudaError_t as int (-1: no kernel).
 int prepare_full_scores(int dtype, int D);
 

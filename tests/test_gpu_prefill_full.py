@@ -168,3 +168,83 @@ def test_full_scores_argument_errors(zb):
         assert e.value.status == zb.ZSM_ERR_INVALID_ARG
     finally:
         cache.close()
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("head_dim,group,T", [(128, 1, 333), (128, 4, 700), (64, 2, 129), (64, 1, 1), (128, 2, 128)])
+def test_prefill_attention_output_lse_and_scores(zb, oracle, dtype, head_dim, group, T):
+    """zsm_prefill_attention: the causal attention output against torch's SDPA in fp64, the rows'
+    log-sum-exp against torch.logsumexp, and the scores it leaves behind against the oracle's
+    full-history prompt pass (one sampled head per sequence when the prompt is long)."""
+    w = wl.Workload("attn", 1, 2, 2 * group, 2, head_dim, dtype, T, 0, T, None, 41)
+    cache = GpuCache(zb, w, [[4, 4]], [[6, 6]], [[1, 1]])
+    try:
+        K, V, Q = wl.prompt(w, 0)
+        dev = "cuda"
+        out = torch.full((w.batch, w.n_q_heads, T, head_dim), float("nan"), dtype=w.torch_dtype, device=dev)
+        lse = torch.full((w.batch, w.n_q_heads, T), float("nan"), dtype=torch.float32, device=dev)
+        scores = torch.full((w.batch, w.n_kv_heads, T), float("nan"), dtype=torch.float32, device=dev)
+        zb.zsm_prefill_attention(cache.h, K.cuda(), V.cuda(), Q.cuda(), T, out, lse, scores)
+        torch.cuda.synchronize()
+        assert cache.status() == 0
+        Kd = K.double().repeat_interleave(group, dim=1)
+        Vd = V.double().repeat_interleave(group, dim=1)
+        Qd = Q.double()
+        ref = torch.nn.functional.scaled_dot_product_attention(Qd, Kd, Vd, is_causal=True)
+        torch.testing.assert_close(out.cpu().double(), ref, atol=2e-3, rtol=1e-2)
+        logits = torch.einsum("bhqd,bhkd->bhqk", Qd, Kd) / np.sqrt(float(head_dim))
+        mask = torch.tril(torch.ones(T, T, dtype=torch.bool))
+        ref_lse = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
+        torch.testing.assert_close(lse.cpu().double(), ref_lse, atol=1e-4, rtol=1e-5)
+        s_gpu = scores.cpu().numpy().astype(np.float64)
+        for b, h in [(0, 0), (1, 1)]:
+            sref = oracle_scores(oracle, cache, K, V, Q, b, h).astype(np.float64)
+            rel = np.abs(s_gpu[b, h] - sref) / np.maximum(np.abs(sref), 1e-30)
+            assert rel.max() <= SCORE_RTOL, f"unit {(b, h)}: relative error {rel.max():.3e}"
+        # without `scores` only the output and the row statistics are produced
+        out2 = torch.empty_like(out)
+        lse2 = torch.empty_like(lse)
+        zb.zsm_prefill_attention(cache.h, K.cuda(), V.cuda(), Q.cuda(), T, out2, lse2)
+        torch.cuda.synchronize()
+        assert torch.equal(out2, out) and torch.equal(lse2, lse)
+    finally:
+        cache.close()
+
+
+def test_prefill_attention_long_prompt(zb):
+    """Many key tiles per query block (the S accumulators, the weight tile, both tile rings and
+    every barrier phase wrap dozens of times), grouped heads; output against SDPA in fp64 on a
+    sample of heads, row sums of the weights through the log-sum-exp."""
+    T, d, G = 4096 + 57, 128, 4
+    w = wl.Workload("attnlong", 1, 1, 2 * G, 2, d, "bf16", T, 0, T, None, 42)
+    cache = GpuCache(zb, w, [[4, 4]], [[6, 6]], [[1, 1]])
+    try:
+        K, V, Q = wl.prompt(w, 0)
+        out = torch.empty(1, 2 * G, T, d, dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty(1, 2 * G, T, dtype=torch.float32, device="cuda")
+        zb.zsm_prefill_attention(cache.h, K.cuda(), V.cuda(), Q.cuda(), T, out, lse)
+        torch.cuda.synchronize()
+        assert cache.status() == 0
+        for hq in (0, 5):
+            hk = hq // G
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                Q[:, hq:hq + 1].double(), K[:, hk:hk + 1].double(), V[:, hk:hk + 1].double(), is_causal=True)
+            torch.testing.assert_close(out[:, hq:hq + 1].cpu().double(), ref, atol=2e-3, rtol=1e-2)
+    finally:
+        cache.close()
+
+
+def test_prefill_attention_argument_errors(zb):
+    w = wl.Workload("attnerr", 1, 1, 2, 2, 64, "f32", 32, 0, 32, None, 43)
+    cache = GpuCache(zb, w, [[4, 4]], [[4, 4]], [[1, 1]])
+    try:
+        K, V, Q = (t.cuda() for t in wl.prompt(w, 0))
+        out = torch.empty_like(Q)
+        lse = torch.empty(1, 2, 32, dtype=torch.float32, device="cuda")
+        with pytest.raises(zb.ZsmError) as e:
+            zb.zsm_prefill_attention(cache.h, K, V, Q, 32, out, lse)
+        assert e.value.status == zb.ZSM_ERR_UNSUPPORTED  # fp32 storage
+        with pytest.raises(ValueError):
+            zb.zsm_prefill_attention(cache.h, K, V, Q, 64, out, lse)  # tensors shorter than T says
+    finally:
+        cache.close()
