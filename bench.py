@@ -374,10 +374,29 @@ def full_history_scores(zb, cache, w, dev, u, stream):
     nres = (T + 127) // 128  # per pass: resident block rb meets 2 rb + 2 streamed tiles of 64 rows
     flop = 2.0 * w.batch * w.n_q_heads * (nres * (nres + 1)) * 128 * 64 * w.head_dim
     tf = measured_tensor_peak()
-    return {"what": "full-history prompt scores (W = T), one layer: row log-sum-exp + decayed column sums",
-            "T": T, "ms_both_passes": ms_both, "ms_column_pass": ms_col,
-            "tflops": 2 * flop / (ms_both * 1e-3) / 1e12, "peak_tflops": tf,
-            "frac": (2 * flop / (ms_both * 1e-3) / 1e12) / tf if tf else None, "bound": "tensor"}
+    res = {"what": "full-history prompt scores (W = T), one layer: row log-sum-exp + decayed column sums",
+           "T": T, "ms_both_passes": ms_both, "ms_column_pass": ms_col,
+           "tflops": 2 * flop / (ms_both * 1e-3) / 1e12, "peak_tflops": tf,
+           "frac": (2 * flop / (ms_both * 1e-3) / 1e12) / tf if tf else None, "bound": "tensor"}
+    # the same scores as a by-product of the prompt's causal attention (output + row statistics +
+    # scores in one call): three passes over Q K^T and one over P V
+    _, Vp, _ = wl.prompt(w, 0, dev, u)
+    out = torch.empty_like(Q)
+    lse_o = torch.empty(w.batch, w.n_q_heads, T, dtype=torch.float32, device=dev)
+    for rep in range(2):
+        ev[0].record(stream)
+        zb.zsm_prefill_attention(cache, Kp, Vp, Q, T, out, lse_o, scores)
+        ev[1].record(stream)
+        zb.zsm_prefill_attention(cache, Kp, Vp, Q, T, out, lse_o)
+        ev[2].record(stream)
+        ev[2].synchronize()
+    ms_all, ms_out = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    res["prefill_attention"] = {
+        "what": "zsm_prefill_attention, one layer: attention output + log-sum-exp (+ scores)",
+        "ms_output_lse_scores": ms_all, "ms_output_lse": ms_out,
+        "tflops": 4 * flop / (ms_all * 1e-3) / 1e12,
+        "frac": (4 * flop / (ms_all * 1e-3) / 1e12) / tf if tf else None}
+    return res
 
 
 def measured_tensor_peak():
