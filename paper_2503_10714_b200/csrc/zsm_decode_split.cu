@@ -187,7 +187,6 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     constexpr int LPR32 = D / 4;
     constexpr int RPW32 = 32 / LPR32;
     constexpr int R32 = kTileBytes / ROWB32;
-    constexpr int RM = kTileBytes / 8;
     constexpr int HDR_K = G * ROWB;  // header tile: q (G rows), k_new, v_new, fusion counts
     constexpr int HDR_V = HDR_K + ROWB;
     constexpr int HDR_W = HDR_V + ROWB;
@@ -206,13 +205,15 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     uint64_t *x_soft = empty_bar + S;  // every rank arrives: softmax partials are in
     uint64_t *x_vict = x_soft + 1;     // rank 0's: every rank's victim candidate is in
     uint64_t *x_done = x_vict + 1;     // rank 0's: partial outputs in, last tiles read
-    uint64_t *l_vict = x_done + 1;     // own consumer warps -> tail warp: candidates are in
-    uint64_t *hdr_bar = l_vict + 1;    // the header (q, k_new, v_new, fusion counts) has landed
+    uint64_t *p_ready = x_done + 1;    // consumer warps -> tail warp: the slice's exponentials are written
+    uint64_t *hdr_bar = p_ready + 1;   // the header (q, k_new, v_new, fusion counts) has landed
+    uint64_t *meta_bar = hdr_bar + 1;  // the slice's scores and positions have landed
     volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(smem + L.flags);
     float *probs = reinterpret_cast<float *>(smem + L.probs);  // [local slot][G]
     float *qf = reinterpret_cast<float *>(smem + L.qf);
     const uint8_t *hdr = smem + L.hdr;
-    float *s_tok_box = reinterpret_cast<float *>(smem + L.mail);
+    float *meta_s = reinterpret_cast<float *>(smem + L.meta);                 // [l_stride] scores
+    int32_t *meta_p = reinterpret_cast<int32_t *>(smem + L.meta) + p.l_stride;  // [l_stride] positions
     const uint4 *kn_raw = reinterpret_cast<const uint4 *>(hdr + HDR_K);
     const uint4 *vn_raw = reinterpret_cast<const uint4 *>(hdr + HDR_V);
     const uint32_t *w_s = reinterpret_cast<const uint32_t *>(hdr + HDR_W);
@@ -220,7 +221,6 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
     float *opart = reinterpret_cast<float *>(smem + L.opart);
     float *redf = reinterpret_cast<float *>(smem + L.redf);
     float *redf2 = redf + kMaxConsumerWarps * 8;
-    uint64_t *red64 = reinterpret_cast<uint64_t *>(smem + L.red64);
     float *xs = reinterpret_cast<float *>(smem + L.xs);  // [rank][16]: max[8], sum[8]
     VictimPost *xv = reinterpret_cast<VictimPost *>(smem + L.xv);
     float *xo = reinterpret_cast<float *>(smem + L.xo);  // [rank][G][D]
@@ -276,9 +276,22 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
             if (br_pad > 0) bulk_g2s(dst + HDR_W, p.base + d.w_off, br_pad * 4u, hdr_bar);
             header_out = true;
         };
-        if (!sp.early) {
+        // scores and positions of the slice: a buffer of their own (the tail warp works on them
+        // while the consumer warps are in the output pass); cache state, like the K tiles
+        auto load_meta = [&]() {
+            const uint32_t n4 = static_cast<uint32_t>((n_loc + 3) & ~3);
+            mbar_arrive_expect_tx(meta_bar, n4 * 8u);
+            if (n4 > 0) {
+                bulk_g2s(meta_s, p.base + d.score_off + (size_t)row_lo * 4, n4 * 4u, meta_bar);
+                bulk_g2s(meta_p, p.base + d.pos_off + (size_t)row_lo * 4, n4 * 4u, meta_bar);
+            }
+        };
+        if (sp.early) {
+            load_meta();
+        } else {
             cluster_wait();
             header();
+            load_meta();
         }
         auto acquire = [&](uint32_t bytes, uint64_t *&bar) -> uint8_t * {
             // the consumers free no stage before they have the header: once the ring is full
@@ -310,14 +323,6 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
             const uint32_t bytes = static_cast<uint32_t>(min(R, row_hi - r0)) * ROWB;
             dst = acquire(bytes, bar);
             if (ok) bulk_g2s(dst, p.base + d.k_off + (size_t)r0 * ROWB, bytes, bar);
-        }
-        for (int j0 = row_lo; j0 < row_hi && ok; j0 += RM) {
-            const uint32_t n4 = static_cast<uint32_t>((min(RM, row_hi - j0) + 3) & ~3);
-            dst = acquire(n4 * 8u, bar);
-            if (ok) {
-                bulk_g2s(dst, p.base + d.score_off + (size_t)j0 * 4, n4 * 4u, bar);
-                bulk_g2s(dst + RM * 4, p.base + d.pos_off + (size_t)j0 * 4, n4 * 4u, bar);
-            }
         }
         for (int r0 = row_lo; r0 < row_hi && ok; r0 += R) {
             const uint32_t bytes = static_cast<uint32_t>(min(R, row_hi - r0)) * ROWB;
@@ -363,19 +368,65 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
         if (sp.early) griddep_wait();
-        // this rank's candidate: the lowest of its consumer warps', posted to rank 0
-        if (!mbar_wait_bounded(l_vict, 0, abort_flag, p.status, WS_VICTIM_LOCAL)) {
+        // D4 + D5 for this rank's slice, while the consumer warps are in the output pass: needs
+        // the slice's exponentials, the cluster's normaliser, and the scores and positions
+        if (!mbar_wait_bounded(p_ready, 0, abort_flag, p.status, WS_VICTIM_LOCAL) ||
+            !mbar_wait_bounded_cluster(x_soft, 0, abort_flag, p.status, WS_SOFTMAX) ||
+            !mbar_wait_bounded(meta_bar, 0, abort_flag, p.status, WS_META)) {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             return;
         }
+        float s_tok = 0.f;  // first score of the new token: its own attention weight (rank 0)
         {
+            float fac[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float M = -INFINITY;
+                for (int r = 0; r < C; ++r) M = fmaxf(M, xs[r * 16 + g]);
+                float Z = 0.f;
+                for (int r = 0; r < C; ++r) Z = fmaf(xs[r * 16 + 8 + g], expf(xs[r * 16 + g] - M), Z);
+                fac[g] = expf(xs[rank * 16 + g] - M) / Z;
+            }
+            const bool evict_l = (n_live == cap);  // the new token does not fit: Alg. 1, overflow branch
+            const int cut = Tpos - d.Bp;           // positions <= cut have left the proximity window
+            float *score_g = reinterpret_cast<float *>(p.base + d.score_off) + row_lo;
             uint64_t key = ~0ull;
             int slot = -1;
-            if (lane < NW) {
-                key = red64[lane * 2];
-                slot = static_cast<int>(static_cast<uint32_t>(red64[lane * 2 + 1]));
+            for (int k = lane; k < n_loc; k += 32) {
+                float pv[G];
+                load_group<G>(probs + k * G, pv);
+                float a = 0.f;
+#pragma unroll
+                for (int g = 0; g < G; ++g) a += pv[g] * fac[g];
+                a *= (1.0f / G);
+                const float s_new = fmaf(p.lambda, meta_s[k], a);  // Eq. (score)
+                score_g[k] = s_new;
+                const int32_t pj = meta_p[k];
+                if (evict_l && pj <= cut) {
+                    const uint64_t kk = (static_cast<uint64_t>(score_order_bits(s_new)) << 32) | (uint32_t)pj;
+                    if (kk < key) {
+                        key = kk;
+                        slot = row_lo + k;
+                    }
+                }
+            }
+            if (rank == 0) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) s_tok += probs[(n_ent - 1) * G + g] * fac[g];
+                s_tok *= (1.0f / G);
+                if (evict_l && d.Bp == 0 && lane == 0) {
+                    const uint64_t kk = (static_cast<uint64_t>(score_order_bits(s_tok)) << 32) | (uint32_t)Tpos;
+                    if (kk < key) {
+                        key = kk;
+                        slot = -2;
+                    }
+                }
             }
             warp_min_key(key, slot);
+            // the new scores are in global memory before rank 0 learns of the candidate (it
+            // overwrites the victim's)
+            fence_cluster();
+            __syncwarp();
             if (lane == 0) {
                 const uint32_t ra = map_to_rank(xv + rank, 0u);
                 st_remote_b64(ra, key);
@@ -407,7 +458,6 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
                 victim_pos = static_cast<int>(static_cast<uint32_t>(best & 0xffffffffull));
             }
         }
-        const float s_tok = *s_tok_box;
         const bool have_victim = evict && victim_slot != -1;
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncwarp();
@@ -752,72 +802,10 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
         }
         mbar_arrive_remote(map_to_rank(x_soft, static_cast<uint32_t>(tid)));
     }
-    if (!mbar_wait_bounded_cluster(x_soft, 0, abort_flag, p.status, WS_SOFTMAX)) return;
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-        float M = -INFINITY;
-        for (int r = 0; r < C; ++r) M = fmaxf(M, xs[r * 16 + g]);
-        float Z = 0.f;
-        for (int r = 0; r < C; ++r) Z = fmaf(xs[r * 16 + 8 + g], expf(xs[r * 16 + g] - M), Z);
-        fac[g] = expf(mx[g] - M) / Z;  // turns this slice's exponentials into attention weights
-    }
-
-    // ---------------- D4 + D5: score update and victim search ----------------
-    const bool evict = (n_live == cap);  // the new token does not fit: Alg. 1, overflow branch
-    const int cut = Tpos - d.Bp;         // positions <= cut have left the proximity window
-    float *score_g = reinterpret_cast<float *>(p.base + d.score_off) + row_lo;
-    uint64_t best = ~0ull;
-    int best_slot = -1;
-    for (int j0 = 0; j0 < n_loc; j0 += RM) {
-        const uint8_t *tile = wait_full(WS_META);
-        if (!tile) return;
-        const int nn = min(RM, n_loc - j0);
-        const float *ts = reinterpret_cast<const float *>(tile);
-        const int32_t *tp = reinterpret_cast<const int32_t *>(tile + RM * 4);
-        for (int k = tid; k < nn; k += NT) {
-            float pv[G];
-            load_group<G>(probs + (j0 + k) * G, pv);
-            float a = 0.f;
-#pragma unroll
-            for (int g = 0; g < G; ++g) a += pv[g] * fac[g];
-            a *= (1.0f / G);
-            const float s_new = fmaf(p.lambda, ts[k], a);  // Eq. (score)
-            score_g[j0 + k] = s_new;
-            const int32_t pj = tp[k];
-            if (evict && pj <= cut) {
-                const uint64_t key = (static_cast<uint64_t>(score_order_bits(s_new)) << 32) | (uint32_t)pj;
-                if (key < best) {
-                    best = key;
-                    best_slot = row_lo + j0 + k;
-                }
-            }
-        }
-        release();
-    }
-    float s_tok = 0.f;  // first score of the new token: its own attention weight (rank 0)
-    if (rank == 0) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) s_tok += probs[(n_ent - 1) * G + g] * fac[g];
-        s_tok *= (1.0f / G);
-    }
-    if (evict) {
-        if (tid == 0 && rank == 0 && d.Bp == 0) {
-            const uint64_t key = (static_cast<uint64_t>(score_order_bits(s_tok)) << 32) | (uint32_t)Tpos;
-            if (key < best) {
-                best = key;
-                best_slot = -2;
-            }
-        }
-        warp_min_key(best, best_slot);
-    }
-    // The warp's candidate goes to the tail warp, which folds the warps' and posts the rank's;
-    // the consumer warps carry on with the V tiles.
-    if (lane == 0) {
-        red64[warp * 2] = best;
-        red64[warp * 2 + 1] = static_cast<uint64_t>(static_cast<uint32_t>(best_slot));
-        if (tid == 0 && rank == 0) *s_tok_box = s_tok;
-        mbar_arrive(l_vict);
-    }
+    // the slice's exponentials are final (un-normalised): the tail warp takes the score update
+    // and the victim search from here (it waits for the cluster's normaliser), the consumer
+    // warps go straight on to the V tiles, which need it only at the very end
+    if (tid == 0) mbar_arrive(p_ready);
 
     // ---------------- D3: output ----------------
     float2 acc2[G][EP2];
@@ -921,6 +909,15 @@ __device__ __forceinline__ void split_body(const SplitParams &sp, uint8_t *smem,
         }
     }
     csync();
+    if (!mbar_wait_bounded_cluster(x_soft, 0, abort_flag, p.status, WS_SOFTMAX)) return;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        float M = -INFINITY;
+        for (int r = 0; r < C; ++r) M = fmaxf(M, xs[r * 16 + g]);
+        float Z = 0.f;
+        for (int r = 0; r < C; ++r) Z = fmaf(xs[r * 16 + 8 + g], expf(xs[r * 16 + g] - M), Z);
+        fac[g] = expf(mx[g] - M) / Z;  // turns this slice's exponentials into attention weights
+    }
     {
         // this rank's share of the output, already normalised, to rank 0
         const T *vn = reinterpret_cast<const T *>(vn_raw);
@@ -983,8 +980,9 @@ __global__ void __launch_bounds__(TWO ? kSplitPairThreads : kSplitThreads, TWO ?
         mbar_init(&bars[2 * S + 1], C);  // victim candidates (used on rank 0)
         // partial outputs, last tiles read (used on rank 0): every posting warp of every rank
         mbar_init(&bars[2 * S + 2], C * split_post_warps(NW, G * D));
-        mbar_init(&bars[2 * S + 3], NW);  // victim candidates of this CTA's consumer warps
+        mbar_init(&bars[2 * S + 3], 1);   // the slice's exponentials are written
         mbar_init(&bars[2 * S + 4], 1);   // header
+        mbar_init(&bars[2 * S + 5], 1);   // scores and positions
         *reinterpret_cast<volatile int32_t *>(smem + L.flags) = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -63,7 +63,7 @@ __host__ __device__ inline int split_l_stride(int cap_max, int br_max, int elem_
 
 // Shared-memory map of one CTA of the split form (byte offsets).
 struct SplitSmem {
-    uint32_t ring, bars, flags, hdr, probs, qf, mail, krs, opart, redf, red64, xs, xv, xo, total;
+    uint32_t ring, bars, flags, hdr, meta, probs, qf, krs, opart, redf, xs, xv, xo, total;
 };
 
 // Bytes of the header a CTA receives after the launch's inputs are known to be ready: q (G rows),
@@ -83,16 +83,15 @@ __host__ __device__ inline SplitSmem split_smem_layout(int stages, int G, int D,
         return at;
     };
     L.ring = take(static_cast<uint32_t>(stages) * kTileBytes);
-    L.bars = take((2u * static_cast<uint32_t>(stages) + 5u) * 8u);
+    L.bars = take((2u * static_cast<uint32_t>(stages) + 6u) * 8u);
     L.flags = take(64u);
     L.hdr = take(split_header_bytes(G, row_bytes, br_max_pad));
+    L.meta = take(static_cast<uint32_t>(l_stride) * 8u);  // the slice's scores, then its positions
     L.probs = take(static_cast<uint32_t>(G) * l_stride * 4u);
     L.qf = take(static_cast<uint32_t>(G) * D * 4u);
-    L.mail = take(decode_mail_bytes(row_bytes, br_max_pad));
     L.krs = take(static_cast<uint32_t>(kr_rows) * D * 4u);
     L.opart = take(static_cast<uint32_t>(consumer_warps) * G * D * 4u);
     L.redf = take(2u * kMaxConsumerWarps * 8u * 4u);
-    L.red64 = take(kMaxConsumerWarps * 16u);
     L.xs = take(kSplitMaxCluster * 2u * 8u * 4u);                       // (max, sum) per rank and head
     L.xv = take(kSplitMaxCluster * 16u);                                // victim candidate per rank
     L.xo = take(static_cast<uint32_t>(cluster) * G * D * 4u);           // partial outputs per rank
