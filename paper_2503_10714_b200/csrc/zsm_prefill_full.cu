@@ -32,6 +32,8 @@
 
 #include <cuda.h>
 
+#include <type_traits>
+
 namespace zsm {
 
 namespace {
@@ -306,31 +308,56 @@ __global__ void __launch_bounds__(kTcThreads, 2)
         const int col0 = jb * kTcRows + ch * 32;
         if (!COLSUM) {
             float bm = -INFINITY;
+            if (diag) {  // only the tile on the diagonal needs the causal mask (warp-uniform branch)
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-                float x = __uint_as_float(v[e]) * scale2;
-                if (diag && col0 + e > row) x = -INFINITY;  // keep key <= query
-                v[e] = __float_as_uint(x);
-                bm = fmaxf(bm, x);
+                for (int e = 0; e < 32; ++e) {
+                    float x = __uint_as_float(v[e]) * scale2;
+                    if (col0 + e > row) x = -INFINITY;  // keep key <= query
+                    v[e] = __float_as_uint(x);
+                    bm = fmaxf(bm, x);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float x = __uint_as_float(v[e]) * scale2;
+                    v[e] = __float_as_uint(x);
+                    bm = fmaxf(bm, x);
+                }
             }
             const float mn = fmaxf(m, bm);
             const float mu = mn == -INFINITY ? 0.f : mn;
-            float sum = z * ex2(m - mu);
+            float sum = z * ex2(m - mu), sum1 = 0.f;  // two chains of additions
 #pragma unroll
-            for (int e = 0; e < 32; ++e) sum += ex2(__uint_as_float(v[e]) - mu);
-            z = sum;
+            for (int e = 0; e < 32; e += 2) {
+                sum += ex2(__uint_as_float(v[e]) - mu);
+                sum1 += ex2(__uint_as_float(v[e + 1]) - mu);
+            }
+            z = sum + sum1;
             m = mn;
         } else {
+            if (diag) {  // only the tile on the diagonal needs the causal mask (warp-uniform branch)
 #pragma unroll
-            for (int e4 = 0; e4 < 8; ++e4) {
-                const float4 o = *reinterpret_cast<const float4 *>(off + ch * 32 + e4 * 4);
-                const float oo[4] = {o.x, o.y, o.z, o.w};
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    const float4 o = *reinterpret_cast<const float4 *>(off + ch * 32 + e4 * 4);
+                    const float oo[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float x = ex2(fmaf(__uint_as_float(v[e4 * 4 + e]), scale2, oo[e]));
-                    if (diag && col0 + e4 * 4 + e < row) x = 0.f;  // keep query >= key
-                    colsum += x;
+                    for (int e = 0; e < 4; ++e) {
+                        float x = ex2(fmaf(__uint_as_float(v[e4 * 4 + e]), scale2, oo[e]));
+                        if (col0 + e4 * 4 + e < row) x = 0.f;  // keep query >= key
+                        colsum += x;
+                    }
                 }
+            } else {
+                float cs1 = 0.f;  // two chains of additions
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    const float4 o = *reinterpret_cast<const float4 *>(off + ch * 32 + e4 * 4);
+                    colsum += ex2(fmaf(__uint_as_float(v[e4 * 4]), scale2, o.x));
+                    cs1 += ex2(fmaf(__uint_as_float(v[e4 * 4 + 1]), scale2, o.y));
+                    colsum += ex2(fmaf(__uint_as_float(v[e4 * 4 + 2]), scale2, o.z));
+                    cs1 += ex2(fmaf(__uint_as_float(v[e4 * 4 + 3]), scale2, o.w));
+                }
+                colsum += cs1;
             }
         }
         }
@@ -437,36 +464,100 @@ __global__ void __launch_bounds__(kTcThreads, 2)
                      : "memory");
 }
 
+// A whole accumulator row: 128 columns of this thread's lane in one load, then the wait.
+__device__ __forceinline__ void tmem_ld128(uint32_t taddr, uint32_t (&v)[128]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x128.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+        "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+        "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, "
+        "%64, %65, %66, %67, %68, %69, %70, %71, %72, %73, %74, %75, %76, %77, %78, %79, "
+        "%80, %81, %82, %83, %84, %85, %86, %87, %88, %89, %90, %91, %92, %93, %94, %95, "
+        "%96, %97, %98, %99, %100, %101, %102, %103, %104, %105, %106, %107, %108, %109, %110, %111, "
+        "%112, %113, %114, %115, %116, %117, %118, %119, %120, %121, %122, %123, %124, %125, %126, %127}, [%128];\n\t"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]),
+          "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]),
+          "=r"(v[40]), "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]),
+          "=r"(v[48]), "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]),
+          "=r"(v[56]), "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63]),
+          "=r"(v[64]), "=r"(v[65]), "=r"(v[66]), "=r"(v[67]), "=r"(v[68]), "=r"(v[69]), "=r"(v[70]), "=r"(v[71]),
+          "=r"(v[72]), "=r"(v[73]), "=r"(v[74]), "=r"(v[75]), "=r"(v[76]), "=r"(v[77]), "=r"(v[78]), "=r"(v[79]),
+          "=r"(v[80]), "=r"(v[81]), "=r"(v[82]), "=r"(v[83]), "=r"(v[84]), "=r"(v[85]), "=r"(v[86]), "=r"(v[87]),
+          "=r"(v[88]), "=r"(v[89]), "=r"(v[90]), "=r"(v[91]), "=r"(v[92]), "=r"(v[93]), "=r"(v[94]), "=r"(v[95]),
+          "=r"(v[96]), "=r"(v[97]), "=r"(v[98]), "=r"(v[99]), "=r"(v[100]), "=r"(v[101]), "=r"(v[102]), "=r"(v[103]),
+          "=r"(v[104]), "=r"(v[105]), "=r"(v[106]), "=r"(v[107]), "=r"(v[108]), "=r"(v[109]), "=r"(v[110]), "=r"(v[111]),
+          "=r"(v[112]), "=r"(v[113]), "=r"(v[114]), "=r"(v[115]), "=r"(v[116]), "=r"(v[117]), "=r"(v[118]), "=r"(v[119]),
+          "=r"(v[120]), "=r"(v[121]), "=r"(v[122]), "=r"(v[123]), "=r"(v[124]), "=r"(v[125]), "=r"(v[126]), "=r"(v[127])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Sixteen 32-bit columns of this thread's lane (32 packed 16-bit weights) into tensor memory.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
+        :
+        : "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
+// Product with the M x K operand in tensor memory (lane = row, a 32-bit column holds two
+// consecutive 16-bit elements of the row) and the N x K operand through a shared-memory descriptor.
+__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t"
+        "}\n"
+        :
+        : "r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
 // ---------------------------------------------------------------------------
 // Causal attention output of the prompt, o_tau = sum_{t <= tau} a^(tau)_t v_t [Eq. (att_score)], from
 // the rows' log-sum-exp of pass 1: with the normaliser known no running maximum is needed, so a
-// tile's weights exp(logit - lse) are final when they are computed.  Per CTA a block of 128
-// queries of one head is resident; for every key tile up to the diagonal
-//   product 1   S = Q K^T            (tcgen05.mma, two accumulators of 128 columns, as above)
-//   epilogue    P = exp2(S * scale - lse) as 16-bit values, written to shared memory in the
-//               K-major 128-byte-swizzled layout the tensor map gives an operand tile
-//   product 2   O += P V             (tcgen05.mma; V's tile, rows = keys, is the N x K operand in
-//               "MN-major" form: N = head dimension contiguous)
-// O is a third accumulator (128 lanes x d columns), read back once at the end.  One warp requests
-// tiles and issues both products, eight warps do the exponentials.  384 (320) tensor-memory
-// columns: one CTA per SM.
+// tile's weights exp(logit - lse) are final when they are computed.  Per CTA two blocks of 128
+// queries of one head are resident, each with a group of four warps of its own; every key and
+// value tile up to the diagonal is fetched once and serves both blocks.  For block g and key tile j
+//   product 1   S_g = Q_g K_j^T      (tcgen05.mma, both operands from shared memory, 128 fp32
+//                                     columns of tensor memory per block)
+//   weights     P_g = exp2(S_g * scale - lse) as 16-bit values, written back into the columns S_g
+//               came from (two weights per 32-bit column; bf16 storage: the high parts in the first
+//               64 columns, the remainders in the other 64)
+//   product 2   O_g += P_g V_j       (tcgen05.mma with the M x K operand in tensor memory; V's tile,
+//               rows = keys, is the N x K operand in "MN-major" form: N = head dimension contiguous)
+// The weights never pass through shared memory, and the two groups work on different products at
+// any time: while one group's exponentials run, the tensor cores multiply for the other.  The
+// products of one block follow one another in issue order on the tensor pipe, which is what lets
+// S_g(j + 1) overwrite the columns P_g(j) was read from.  One thread requests tiles and issues
+// every product.  2 x 128 (S) + 2 x d (O) tensor-memory columns: one CTA per SM.
 // ---------------------------------------------------------------------------
 constexpr int kAoThreads = kTcEpiThreads + 32;
-enum : int32_t { WA_S = 51, WA_P = 52, WA_PFREE = 53, WA_K = 54, WA_V = 55, WA_VFREE = 56, WA_SFREE = 57, WA_O = 58, WA_Q = 59 };
+constexpr int kAoKStages = 3;  // key tiles in shared memory
+constexpr int kAoVStages = 2;  // value tiles
+enum : int32_t { WA_S = 51, WA_P = 52, WA_K = 54, WA_V = 55, WA_VFREE = 56, WA_O = 58, WA_Q = 59 };
 
 template <int D>
 struct AoSmem {
     static constexpr int KB = D / kTcKBlock;
     static constexpr int KBLOCK = kTcRows * 128;
     static constexpr int TILE = KB * KBLOCK;          // Q, K or V tile
-    static constexpr int PTILE = 2 * KBLOCK;          // 128 queries x 128 keys, 16 bit
-    static constexpr int q = 0;
-    static constexpr int k = TILE;                    // two stages
-    static constexpr int v = k + 2 * TILE;            // two stages
-    static constexpr int pw = v + 2 * TILE;           // the weights of the tile in hand
-    static constexpr int bars = pw + 2 * PTILE;       // high parts, then (bf16 only) the remainders
+    static constexpr int q = 0;                       // two query blocks
+    static constexpr int k = 2 * TILE;
+    static constexpr int v = k + kAoKStages * TILE;
+    static constexpr int bars = v + kAoVStages * TILE;
     static constexpr int total = bars + 256 + 1024;   // + slack to align the base to 1 KiB
-    static constexpr int tmem_cols = 512;             // 2 x 128 (S) + D (O), rounded up to a power of two
+    static constexpr int tmem_cols = 512;             // 2 x 128 (S) + 2 x D (O), a power of two
 };
 
 // V tile as the N x K operand with N (head dimension) contiguous: 64 elements per 128-byte row,
@@ -492,40 +583,43 @@ __global__ void __launch_bounds__(kAoThreads, 1)
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t *q_bar = reinterpret_cast<uint64_t *>(smem + L::bars);
-    uint64_t *k_full = q_bar + 1;      // [2] key tile landed
-    uint64_t *v_full = k_full + 2;     // [2] value tile landed
-    uint64_t *v_free = v_full + 2;     // [2] product 2 done with the value tile (and with the weights)
-    uint64_t *s_ready = v_free + 2;    // [2] product 1 complete
-    uint64_t *s_free = s_ready + 2;    // [2] accumulator read by the eight warps
-    uint64_t *p_ready = s_free + 2;    // weights written by the eight warps
-    uint64_t *p_free = p_ready + 1;    // product 2 has read the weights
-    uint64_t *o_done = p_free + 1;     // every product complete
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(o_done + 1);
+    uint64_t *k_full = q_bar + 1;               // [3] key tile landed
+    uint64_t *v_full = k_full + kAoKStages;     // [2] value tile landed
+    uint64_t *v_free = v_full + kAoVStages;     // [2] both blocks' product 2 done with the value tile
+    uint64_t *s_ready = v_free + kAoVStages;    // [2] block g's product 1 complete
+    uint64_t *p_ready = s_ready + 2;            // [2] block g's weights written by its four warps
+    uint64_t *o_done = p_ready + 2;             // [2] block g's last product complete
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(o_done + 2);
     volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(tmem_slot + 2);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Tn = p.T, G = p.G;
     const int nb = (Tn + kTcRows - 1) / kTcRows;
-    const int rb = nb - 1 - blockIdx.x;  // the longest blocks first
+    const int nb2 = (nb + 1) / 2;
+    const int rb2 = nb2 - 1 - blockIdx.x;  // the longest pairs of blocks first
     const int b = blockIdx.y / (p.n_kv_heads * G);
     const int hq = blockIdx.y % (p.n_kv_heads * G);
     const int zk = b * p.n_kv_heads + hq / G;
     const int zq = b * p.n_kv_heads * G + hq;
-    const int n_tiles = rb + 1;
+    // block g holds queries 128 (2 rb2 + g) ..; it walks the key tiles 0 .. 2 rb2 + g.  The second
+    // block of the last pair may lie past the prompt's end: then it has no tile at all.
+    const int n0 = 2 * rb2 + 1;
+    const int n1 = (2 * rb2 + 1 < nb) ? 2 * rb2 + 2 : 0;
+    const int nmax = n1 > n0 ? n1 : n0;
     const float scale2 = p.scale * kLog2e;
 
     if (tid == 0) {
         mbar_init(q_bar, 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&k_full[s], 1);
+        for (int s = 0; s < kAoKStages; ++s) mbar_init(&k_full[s], 1);
+        for (int s = 0; s < kAoVStages; ++s) {
             mbar_init(&v_full[s], 1);
             mbar_init(&v_free[s], 1);
-            mbar_init(&s_ready[s], 1);
-            mbar_init(&s_free[s], kTcEpiThreads / 32);
         }
-        mbar_init(p_ready, kTcEpiThreads / 32);
-        mbar_init(p_free, 1);
-        mbar_init(o_done, 1);
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(&s_ready[g], 1);
+            mbar_init(&p_ready[g], 4);
+            mbar_init(&o_done[g], 1);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -541,7 +635,7 @@ __global__ void __launch_bounds__(kAoThreads, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_o = tmem_base + 2 * kTcRows;
+    const uint32_t tmem_o = tmem_base + 2 * kTcRows;  // O_g at tmem_o + g * D
 
     const uint32_t f = E::kIsBf16 ? 1u : 0u;
     const uint32_t idesc_s = (1u << 4) | (f << 7) | (f << 10) | ((kTcRows >> 3) << 17) | ((kTcRows >> 4) << 24);
@@ -559,141 +653,166 @@ __global__ void __launch_bounds__(kAoThreads, 1)
                 for (int kb = 0; kb < L::KB; ++kb)
                     tma_load_3d(dst + kb * L::KBLOCK, map, kb * kTcKBlock, jb * kTcRows, z, bar);
             };
-            load_tile(smem + L::q, &map_q, zq, rb, q_bar);
-            for (int i = 0; i < 2 && i < n_tiles; ++i) {
-                load_tile(smem + L::k + i * L::TILE, &map_k, zk, i, &k_full[i]);
-                load_tile(smem + L::v + i * L::TILE, &map_v, zk, i, &v_full[i]);
-            }
-            // product 2 of tile t: needs its weights and its value tile
-            auto issue_pv = [&](int t) {
-                if (!mbar_wait_bounded(p_ready, t & 1u, abort_flag, p.status, WA_P)) return false;
-                // the weights exist, so product 1 of tile t is complete: its key stage is free
-                if (t + 2 < n_tiles)
-                    load_tile(smem + L::k + (t & 1) * L::TILE, &map_k, zk, t + 2, &k_full[t & 1]);
-                if (!mbar_wait_bounded(&v_full[t & 1], (t >> 1) & 1u, abort_flag, p.status, WA_V)) return false;
-                tc_fence_after();
-                const uint8_t *vt = smem + L::v + (t & 1) * L::TILE;
+            // both query blocks on one barrier (rows past the prompt's end read as zero)
+            mbar_arrive_expect_tx(q_bar, 2 * L::TILE);
+            for (int g = 0; g < 2; ++g)
 #pragma unroll
-                for (int ks = 0; ks < kTcRows / 16; ++ks) {
-                    const int o = (ks / 4) * L::KBLOCK + (ks % 4) * 32;  // 16 keys = 32 bytes of a weight row
-                    umma_f16_ss(tmem_o, umma_desc_sw128(smem + L::pw + o), umma_desc_v_mn<D>(vt, ks), idesc_o,
-                                (t > 0 || ks > 0) ? 1u : 0u);
-                    if constexpr (kSplitW)
-                        umma_f16_ss(tmem_o, umma_desc_sw128(smem + L::pw + L::PTILE + o), umma_desc_v_mn<D>(vt, ks),
-                                    idesc_o, 1u);
-                }
-                umma_commit(p_free);
-                umma_commit(&v_free[t & 1]);
-                return true;
-            };
-            ok = mbar_wait_bounded(q_bar, 0, abort_flag, p.status, WA_Q);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                ok = mbar_wait_bounded(&k_full[j & 1], (j >> 1) & 1u, abort_flag, p.status, WA_K);
-                if (ok && j >= 2)
-                    ok = mbar_wait_bounded(&s_free[j & 1], ((j - 2) >> 1) & 1u, abort_flag, p.status, WA_SFREE);
-                if (!ok) break;
-                tc_fence_after();
-                const uint8_t *kt = smem + L::k + (j & 1) * L::TILE;
+                for (int kb = 0; kb < L::KB; ++kb)
+                    tma_load_3d(smem + L::q + g * L::TILE + kb * L::KBLOCK, &map_q, kb * kTcKBlock,
+                                (2 * rb2 + g) * kTcRows, zq, q_bar);
+            for (int i = 0; i < kAoKStages && i < nmax; ++i)
+                load_tile(smem + L::k + i * L::TILE, &map_k, zk, i, &k_full[i]);
+            for (int i = 0; i < kAoVStages && i < nmax; ++i)
+                load_tile(smem + L::v + i * L::TILE, &map_v, zk, i, &v_full[i]);
+            // product 1 of block g with key tile j (its stage has landed)
+            auto issue_s = [&](int g, int j) {
+                const uint8_t *kt = smem + L::k + (j % kAoKStages) * L::TILE;
+                const uint8_t *qt = smem + L::q + g * L::TILE;
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
-                    const int o = (ks / 4) * L::KBLOCK + (ks % 4) * 32;
-                    umma_f16_ss(tmem_base + (j & 1) * kTcRows, umma_desc_sw128(smem + L::q + o),
-                                umma_desc_sw128(kt + o), idesc_s, ks > 0);
+                    const int o = (ks / 4) * L::KBLOCK + (ks % 4) * 32;  // 16 elements = 32 bytes on
+                    umma_f16_ss(tmem_base + g * kTcRows, umma_desc_sw128(qt + o), umma_desc_sw128(kt + o), idesc_s,
+                                ks > 0);
                 }
-                umma_commit(&s_ready[j & 1]);
-                if (j >= 1) ok = issue_pv(j - 1);
-                if (ok && j >= 2) {
-                    // value stage of tile j - 2 (the one tile j will use) is free once its product is done
-                    ok = mbar_wait_bounded(&v_free[j & 1], ((j - 2) >> 1) & 1u, abort_flag, p.status, WA_VFREE);
-                    if (ok) load_tile(smem + L::v + (j & 1) * L::TILE, &map_v, zk, j, &v_full[j & 1]);
+                umma_commit(&s_ready[g]);
+            };
+            // product 2 of block g with value tile j: the weights sit where S_g was
+            auto issue_pv = [&](int g, int j) {
+                const uint8_t *vt = smem + L::v + (j % kAoVStages) * L::TILE;
+                const uint32_t pw = tmem_base + g * kTcRows;
+#pragma unroll
+                for (int ks = 0; ks < kTcRows / 16; ++ks) {  // 16 keys = 8 columns of packed weights
+                    umma_f16_ts(tmem_o + g * D, pw + ks * 8, umma_desc_v_mn<D>(vt, ks), idesc_o,
+                                (j > 0 || ks > 0) ? 1u : 0u);
+                    if constexpr (kSplitW)
+                        umma_f16_ts(tmem_o + g * D, pw + 64 + ks * 8, umma_desc_v_mn<D>(vt, ks), idesc_o, 1u);
                 }
+            };
+            ok = mbar_wait_bounded(q_bar, 0, abort_flag, p.status, WA_Q) &&
+                 mbar_wait_bounded(&k_full[0], 0, abort_flag, p.status, WA_K);
+            if (ok) {
+                tc_fence_after();
+                issue_s(0, 0);
+                if (n1 > 0) issue_s(1, 0);
             }
-            if (ok) ok = issue_pv(n_tiles - 1);
-            if (ok) umma_commit(o_done);
+            for (int j = 0; j < nmax && ok; ++j) {
+                if (j >= 1) {
+                    // the products of tile j - 1 are done with their value stage: tile j + 1 goes there
+                    ok = mbar_wait_bounded(&v_free[(j - 1) % kAoVStages], ((j - 1) / kAoVStages) & 1u, abort_flag,
+                                           p.status, WA_VFREE);
+                    if (ok && j + 1 < nmax)
+                        load_tile(smem + L::v + ((j + 1) % kAoVStages) * L::TILE, &map_v, zk, j + 1,
+                                  &v_full[(j + 1) % kAoVStages]);
+                }
+                if (ok)
+                    ok = mbar_wait_bounded(&v_full[j % kAoVStages], (j / kAoVStages) & 1u, abort_flag, p.status, WA_V);
+                bool k_next = false;
+                for (int g = 0; g < 2 && ok; ++g) {
+                    const int n = g ? n1 : n0;
+                    if (j >= n) continue;
+                    ok = mbar_wait_bounded(&p_ready[g], j & 1u, abort_flag, p.status, WA_P);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(g, j);
+                    if (j + 1 == n) umma_commit(&o_done[g]);
+                    if (j + 1 < n) {
+                        if (!k_next) {
+                            ok = mbar_wait_bounded(&k_full[(j + 1) % kAoKStages], ((j + 1) / kAoKStages) & 1u,
+                                                   abort_flag, p.status, WA_K);
+                            if (!ok) break;
+                            tc_fence_after();
+                            k_next = true;
+                        }
+                        issue_s(g, j + 1);
+                    }
+                }
+                if (!ok) break;
+                umma_commit(&v_free[j % kAoVStages]);
+                // both blocks have turned S(j) into weights, so product 1 of tile j is complete and
+                // its key stage is free
+                if (j + kAoKStages < nmax)
+                    load_tile(smem + L::k + (j % kAoKStages) * L::TILE, &map_k, zk, j + kAoKStages,
+                              &k_full[j % kAoKStages]);
+            }
             if (!ok) {
+                // copies that were requested may still land: give them time before the memory goes away
                 const uint64_t t0 = global_timer_ns();
                 while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
     } else {
-        // eight warps: accumulator lanes 32 quad .., columns 64 cq ..
-        const int quad = warp & 3, cq = warp >> 2;
+        // two groups of four warps: group g owns query block g; accumulator lanes 32 quad ..
+        const int g = warp >> 2, quad = warp & 3;
+        const int n = g ? n1 : n0;
+        const int qt = 2 * rb2 + g;  // this block's query tile = its diagonal key tile
         const int rloc = quad * 32 + lane;
-        const int row = rb * kTcRows + rloc;
-        const float lse2 = row < Tn ? p.lse[(size_t)zq * Tn + row] * kLog2e : 0.f;
-        uint8_t *prow = smem + L::pw + cq * L::KBLOCK + rloc * 128;
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            const int buf = j & 1;
-            if (!mbar_wait_bounded(&s_ready[buf], (j >> 1) & 1u, abort_flag, p.status, WA_S)) {
+        const int row = qt * kTcRows + rloc;
+        const float lse2 = (n > 0 && row < Tn) ? p.lse[(size_t)zq * Tn + row] * kLog2e : 0.f;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const uint32_t s_addr = lane_base + g * kTcRows;
+        for (int j = 0; j < n && ok; ++j) {
+            if (!mbar_wait_bounded(&s_ready[g], j & 1u, abort_flag, p.status, WA_S)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
-            const bool diag = j == rb;
-            uint32_t w[32];  // 64 weights of this thread's row, packed in pairs
-            uint32_t wl[kSplitW ? 32 : 1];  // their remainders
+            uint32_t v[128];  // this thread's row of S: 128 keys
+            tmem_ld128(s_addr, v);
+            // only the tile on the diagonal needs the causal mask: a warp-uniform branch between
+            // two copies of the loop
+            auto weights = [&](auto masked) {
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kTcRows + cq * 64 + c * 32, v);
-                if (c == 1) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&s_free[buf]);
-                }
-                const int col0 = j * kTcRows + cq * 64 + c * 32;
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t w[16];                  // 32 weights, packed in pairs
+                    uint32_t wl[kSplitW ? 16 : 1];   // their remainders
+                    const int col0 = j * kTcRows + c * 32;
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float x0 = ex2(fmaf(__uint_as_float(v[e]), scale2, -lse2));
-                    float x1 = ex2(fmaf(__uint_as_float(v[e + 1]), scale2, -lse2));
-                    if (row >= Tn || (diag && col0 + e > row)) x0 = 0.f;       // keep key <= query
-                    if (row >= Tn || (diag && col0 + e + 1 > row)) x1 = 0.f;
-                    if constexpr (E::kIsBf16) {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
-                        const float2 hb = __bfloat1622float2(h);
-                        const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - hb.x, x1 - hb.y);
-                        w[c * 16 + e / 2] = *reinterpret_cast<const uint32_t *>(&h);
-                        wl[c * 16 + e / 2] = *reinterpret_cast<const uint32_t *>(&l);
-                    } else {
-                        const __half2 h = __floats2half2_rn(x0, x1);
-                        w[c * 16 + e / 2] = *reinterpret_cast<const uint32_t *>(&h);
+                    for (int e = 0; e < 32; e += 2) {
+                        float x0 = ex2(fmaf(__uint_as_float(v[c * 32 + e]), scale2, -lse2));
+                        float x1 = ex2(fmaf(__uint_as_float(v[c * 32 + e + 1]), scale2, -lse2));
+                        if constexpr (decltype(masked)::value) {
+                            if (col0 + e > row) x0 = 0.f;  // keep key <= query
+                            if (col0 + e + 1 > row) x1 = 0.f;
+                        }
+                        if constexpr (E::kIsBf16) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                            const float2 hb = __bfloat1622float2(h);
+                            const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - hb.x, x1 - hb.y);
+                            w[e / 2] = *reinterpret_cast<const uint32_t *>(&h);
+                            wl[e / 2] = *reinterpret_cast<const uint32_t *>(&l);
+                        } else {
+                            const __half2 h = __floats2half2_rn(x0, x1);
+                            w[e / 2] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
                     }
+                    // the whole row is in registers, so its columns can be overwritten
+                    tmem_st16(s_addr + c * 16, w);
+                    if constexpr (kSplitW) tmem_st16(s_addr + 64 + c * 16, wl);
                 }
-            }
-            // the weights of the tile before this one have been multiplied
-            if (j >= 1 && !mbar_wait_bounded(p_free, (j - 1) & 1u, abort_flag, p.status, WA_PFREE)) {
-                ok = false;
-                break;
-            }
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch)  // 16-byte chunk ch of the row sits at chunk ch ^ (row % 8)
-            {
-                *reinterpret_cast<uint4 *>(prow + ((ch ^ (rloc & 7)) << 4)) =
-                    make_uint4(w[4 * ch], w[4 * ch + 1], w[4 * ch + 2], w[4 * ch + 3]);
-                if constexpr (kSplitW)
-                    *reinterpret_cast<uint4 *>(prow + L::PTILE + ((ch ^ (rloc & 7)) << 4)) =
-                        make_uint4(wl[4 * ch], wl[4 * ch + 1], wl[4 * ch + 2], wl[4 * ch + 3]);
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            };
+            if (j == qt)
+                weights(std::true_type{});
+            else
+                weights(std::false_type{});
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_ready);
+            if (lane == 0) mbar_arrive(&p_ready[g]);
         }
-        if (ok && mbar_wait_bounded(o_done, 0, abort_flag, p.status, WA_O)) {
+        if (n > 0 && ok && mbar_wait_bounded(&o_done[g], 0, abort_flag, p.status, WA_O)) {
             tc_fence_after();
             T *orow = static_cast<T *>(out_ptr) + ((size_t)zq * Tn + row) * D;
 #pragma unroll
-            for (int c = 0; c < D / 64; ++c) {
-                // the eight warps split the d columns: half cq takes columns cq * D/2 ..
-                uint32_t v[32];
-                const int col = cq * (D / 2) + c * 32;
-                tmem_ld32(tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + col, v);
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(lane_base + 2 * kTcRows + g * D + c * 32, o);
                 if (row < Tn) {
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
                         uint32_t pk[4];
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            const float a0 = __uint_as_float(v[e + 2 * k]), a1 = __uint_as_float(v[e + 2 * k + 1]);
+                            const float a0 = __uint_as_float(o[e + 2 * k]), a1 = __uint_as_float(o[e + 2 * k + 1]);
                             if constexpr (E::kIsBf16) {
                                 const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
                                 pk[k] = *reinterpret_cast<const uint32_t *>(&h);
@@ -702,7 +821,7 @@ __global__ void __launch_bounds__(kAoThreads, 1)
                                 pk[k] = *reinterpret_cast<const uint32_t *>(&h);
                             }
                         }
-                        *reinterpret_cast<uint4 *>(orow + col + e) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4 *>(orow + c * 32 + e) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
             }
@@ -801,7 +920,7 @@ int launch_attn_one(const FullScoreParams &p, const void *V, void *out, cudaStre
         !make_map(&map_q, p.Q, p.batch * p.n_kv_heads * p.G, p.T, D, Elem<T>::kIsBf16))
         return static_cast<int>(cudaErrorInvalidValue);
     const int nres = (p.T + kTcRows - 1) / kTcRows;
-    const dim3 grid(nres, p.batch * p.n_kv_heads * p.G);
+    const dim3 grid((nres + 1) / 2, p.batch * p.n_kv_heads * p.G);  // two query blocks per CTA
     attn_out_tc_kernel<T, D><<<grid, kAoThreads, AoSmem<D>::total, stream>>>(p, out, map_k, map_v, map_q);
     return static_cast<int>(cudaGetLastError());
 }
