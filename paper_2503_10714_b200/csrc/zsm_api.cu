@@ -826,18 +826,19 @@ zsm_status_t zsm_prefill_attention(zsm_cache_t *c, const void *K, const void *V,
     p.lambda = c->lambda;
     p.scale = c->scale;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    // row statistics first (and, when asked for, the decayed column sums from them) ...
+    // one pass gives the output and the rows' log-sum-exp ...
     p.lse = nullptr;
     p.lse_out = lse;
-    p.scores = scores;
-    int rc = scores ? launch_full_scores(c->s.dtype, c->s.D, p, cs)
-                    : launch_row_statistics(c->s.dtype, c->s.D, p, cs);
+    p.scores = nullptr;
+    int rc = launch_attention_output(c->s.dtype, c->s.D, p, V, out, cs);
     if (rc == -1) return ZSM_ERR_UNSUPPORTED;
     if (rc != 0) return ZSM_ERR_CUDA;
-    // ... then the output, whose weights exp(logit - lse) need no running maximum
+    if (!scores) return ZSM_OK;
+    // ... from which the decayed column sums follow
     p.lse = lse;
     p.lse_out = nullptr;
-    rc = launch_attention_output(c->s.dtype, c->s.D, p, V, out, cs);
+    p.scores = scores;
+    rc = launch_full_scores(c->s.dtype, c->s.D, p, cs);
     if (rc == -1) return ZSM_ERR_UNSUPPORTED;
     return rc == 0 ? ZSM_OK : ZSM_ERR_CUDA;
 }

@@ -508,6 +508,16 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         : "memory");
 }
 
+// Thirty-two 32-bit columns of this thread's lane into tensor memory.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
+        :
+        : "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+
 // Product with the M x K operand in tensor memory (lane = row, a 32-bit column holds two
 // consecutive 16-bit elements of the row) and the N x K operand through a shared-memory descriptor.
 __device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc,
@@ -524,23 +534,27 @@ __device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, ui
 }
 
 // ---------------------------------------------------------------------------
-// Causal attention output of the prompt, o_tau = sum_{t <= tau} a^(tau)_t v_t [Eq. (att_score)], from
-// the rows' log-sum-exp of pass 1: with the normaliser known no running maximum is needed, so a
-// tile's weights exp(logit - lse) are final when they are computed.  Per CTA two blocks of 128
-// queries of one head are resident, each with a group of four warps of its own; every key and
-// value tile up to the diagonal is fetched once and serves both blocks.  For block g and key tile j
+// Causal attention of the prompt in one pass: o_tau = sum_{t <= tau} a^(tau)_t v_t [Eq. (att_score)]
+// and the log-sum-exp of every query's row.  Per CTA two blocks of 128 queries of one head are
+// resident, each with a group of four warps of its own; every key and value tile up to the
+// diagonal is fetched once and serves both blocks.  For block g and key tile j
 //   product 1   S_g = Q_g K_j^T      (tcgen05.mma, both operands from shared memory, 128 fp32
 //                                     columns of tensor memory per block)
-//   weights     P_g = exp2(S_g * scale - lse) as 16-bit values, written back into the columns S_g
-//               came from (two weights per 32-bit column; bf16 storage: the high parts in the first
-//               64 columns, the remainders in the other 64)
+//   weights     a thread owns one query row: P_g = exp2(S_g * scale - m_ref) as 16-bit values,
+//               written back into the columns S_g came from (two weights per 32-bit column; bf16
+//               storage: the high parts in the first 64 columns, the remainders in the other 64),
+//               and their fp32 sum.  m_ref follows the row's running maximum lazily: it moves
+//               only when a tile's maximum exceeds it by more than 8 (weights stay below 2^8),
+//               and then the thread rescales its row of O_g in tensor memory and its sum
 //   product 2   O_g += P_g V_j       (tcgen05.mma with the M x K operand in tensor memory; V's tile,
 //               rows = keys, is the N x K operand in "MN-major" form: N = head dimension contiguous)
-// The weights never pass through shared memory, and the two groups work on different products at
-// any time: while one group's exponentials run, the tensor cores multiply for the other.  The
-// products of one block follow one another in issue order on the tensor pipe, which is what lets
-// S_g(j + 1) overwrite the columns P_g(j) was read from.  One thread requests tiles and issues
-// every product.  2 x 128 (S) + 2 x d (O) tensor-memory columns: one CTA per SM.
+// At the end o = O_g / sum and lse = m_ref + log2(sum).  The weights never pass through shared
+// memory, and the two groups work on different products at any time: while one group's
+// exponentials run, the tensor cores multiply for the other.  The products of one block follow one
+// another in issue order on the tensor pipe, which is what lets S_g(j + 1) overwrite the columns
+// P_g(j) was read from, and what makes O_g quiescent between "S_g(j) complete" and this group's
+// "weights written".  One thread requests tiles and issues every product.  2 x 128 (S) + 2 x d (O)
+// tensor-memory columns: one CTA per SM.
 // ---------------------------------------------------------------------------
 constexpr int kAoThreads = kTcEpiThreads + 32;
 constexpr int kAoKStages = 3;  // key tiles in shared memory
@@ -747,33 +761,80 @@ __global__ void __launch_bounds__(kAoThreads, 1)
         const int qt = 2 * rb2 + g;  // this block's query tile = its diagonal key tile
         const int rloc = quad * 32 + lane;
         const int row = qt * kTcRows + rloc;
-        const float lse2 = (n > 0 && row < Tn) ? p.lse[(size_t)zq * Tn + row] * kLog2e : 0.f;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const uint32_t s_addr = lane_base + g * kTcRows;
+        const uint32_t o_addr = lane_base + 2 * kTcRows + g * D;
+        // Running softmax of this thread's row, log2 domain: the weights are taken against `m_ref`,
+        // which follows the row's maximum lazily -- it moves only when a tile's maximum exceeds it
+        // by more than 2^8 (so weights stay below 256, within fp16), and then the row of O and
+        // the running sum are rescaled.  After the first tiles that is rare.
+        float m_ref = -INFINITY, l0 = 0.f, l1 = 0.f;
         for (int j = 0; j < n && ok; ++j) {
             if (!mbar_wait_bounded(&s_ready[g], j & 1u, abort_flag, p.status, WA_S)) {
                 ok = false;
                 break;
             }
+            // product 1 of tile j was issued behind product 2 of tile j - 1, so O_g is at rest
+            // until this group announces its weights
             tc_fence_after();
             uint32_t v[128];  // this thread's row of S: 128 keys
             tmem_ld128(s_addr, v);
             // only the tile on the diagonal needs the causal mask: a warp-uniform branch between
-            // two copies of the loop
-            auto weights = [&](auto masked) {
+            // two copies of the loops.  Keys past `lim` (tile-relative) are masked.
+            const bool diag = j == qt;
+            const int lim = row - j * kTcRows;
+            float mx = -INFINITY, mx1 = -INFINITY;
+            if (diag || scale2 <= 0.f) {
+#pragma unroll
+                for (int e = 0; e < 128; ++e) {
+                    float x = __uint_as_float(v[e]) * scale2;
+                    if (diag && e > lim) x = -INFINITY;  // keep key <= query
+                    v[e] = __float_as_uint(x);
+                    mx = fmaxf(mx, x);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 128; e += 2) {
+                    mx = fmaxf(mx, __uint_as_float(v[e]));
+                    mx1 = fmaxf(mx1, __uint_as_float(v[e + 1]));
+                }
+                mx = fmaxf(mx, mx1) * scale2;
+            }
+            const bool move = mx > m_ref + 8.f;  // always on the first tile
+            if (__any_sync(0xffffffffu, move)) {
+                const float m_new = move ? mx : m_ref;
+                const float fac = !move ? 1.f : (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_new));
+                l0 *= fac;
+                l1 *= fac;
+                m_ref = m_new;
+                if (j > 0) {
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(o_addr + c * 32, o);
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fac);
+                        tmem_st32(o_addr + c * 32, o);
+                    }
+                }
+            }
+            auto weights = [&](auto scaled) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t w[16];                  // 32 weights, packed in pairs
                     uint32_t wl[kSplitW ? 16 : 1];   // their remainders
-                    const int col0 = j * kTcRows + c * 32;
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
-                        float x0 = ex2(fmaf(__uint_as_float(v[c * 32 + e]), scale2, -lse2));
-                        float x1 = ex2(fmaf(__uint_as_float(v[c * 32 + e + 1]), scale2, -lse2));
-                        if constexpr (decltype(masked)::value) {
-                            if (col0 + e > row) x0 = 0.f;  // keep key <= query
-                            if (col0 + e + 1 > row) x1 = 0.f;
+                        float x0, x1;
+                        if constexpr (decltype(scaled)::value) {  // v holds scaled, masked logits
+                            x0 = ex2(__uint_as_float(v[c * 32 + e]) - m_ref);
+                            x1 = ex2(__uint_as_float(v[c * 32 + e + 1]) - m_ref);
+                        } else {
+                            x0 = ex2(fmaf(__uint_as_float(v[c * 32 + e]), scale2, -m_ref));
+                            x1 = ex2(fmaf(__uint_as_float(v[c * 32 + e + 1]), scale2, -m_ref));
                         }
+                        l0 += x0;
+                        l1 += x1;
                         if constexpr (E::kIsBf16) {
                             const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
                             const float2 hb = __bfloat1622float2(h);
@@ -790,7 +851,7 @@ __global__ void __launch_bounds__(kAoThreads, 1)
                     if constexpr (kSplitW) tmem_st16(s_addr + 64 + c * 16, wl);
                 }
             };
-            if (j == qt)
+            if (diag || scale2 <= 0.f)
                 weights(std::true_type{});
             else
                 weights(std::false_type{});
@@ -801,18 +862,22 @@ __global__ void __launch_bounds__(kAoThreads, 1)
         }
         if (n > 0 && ok && mbar_wait_bounded(&o_done[g], 0, abort_flag, p.status, WA_O)) {
             tc_fence_after();
+            const float l = l0 + l1;
+            const float inv = 1.0f / l;  // the key at position 0 is visible to every query: l > 0
+            if (row < Tn) p.lse_out[(size_t)zq * Tn + row] = (m_ref + log2f(l)) * kLn2;
             T *orow = static_cast<T *>(out_ptr) + ((size_t)zq * Tn + row) * D;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
-                tmem_ld32(lane_base + 2 * kTcRows + g * D + c * 32, o);
+                tmem_ld32(o_addr + c * 32, o);
                 if (row < Tn) {
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
                         uint32_t pk[4];
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            const float a0 = __uint_as_float(o[e + 2 * k]), a1 = __uint_as_float(o[e + 2 * k + 1]);
+                            const float a0 = __uint_as_float(o[e + 2 * k]) * inv;
+                            const float a1 = __uint_as_float(o[e + 2 * k + 1]) * inv;
                             if constexpr (E::kIsBf16) {
                                 const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
                                 pk[k] = *reinterpret_cast<const uint32_t *>(&h);

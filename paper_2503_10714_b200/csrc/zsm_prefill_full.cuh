@@ -23,8 +23,8 @@ struct FullScoreParams {
 int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t stream);
 // The first pass alone: every query row's log-sum-exp into p.lse_out.
 int launch_row_statistics(int dtype, int D, const FullScoreParams &p, cudaStream_t stream);
-// Causal attention output of the prompt from the rows' log-sum-exp (p.lse, required):
-// out [batch][n_q_heads][T][d] in the storage dtype; V [batch][n_kv_heads][T][d].
+// Causal attention of the prompt in one pass: out [batch][n_q_heads][T][d] in the storage dtype and
+// every query row's log-sum-exp into p.lse_out (required; p.lse is not read); V [batch][n_kv_heads][T][d].
 int launch_attention_output(int dtype, int D, const FullScoreParams &p, const void *V, void *out,
                             cudaStream_t stream);
 // Raises the kernels' dynamic shared-memory limit; returns a cudaError_t as int (-1: no kernel).
