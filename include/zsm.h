@@ -218,9 +218,9 @@ zsm_status_t zsm_prefill_scores_full(zsm_cache_t *c, const void *K, const void *
  * history]: out[b][hq][tau] = sum_{t <= tau} a^(tau)_t v_t, the rows' log-sum-exp, and -- when
  * `scores` is given -- the full-history scores of zsm_prefill_scores_full, ready for
  * zsm_prefill_compress(scores = ...).  A model that runs this as its prefill attention needs no
- * separate scoring pass.  Tensor cores throughout (tcgen05): row statistics, then the output as
- * two products per key tile (Q K^T; weights exp(logit - lse) as 16-bit values times V), then the
- * decayed column sums.
+ * separate scoring pass.  Tensor cores throughout (tcgen05): one pass for the output and the
+ * rows' log-sum-exp (two products per key tile: Q K^T; 16-bit weights of a running softmax times
+ * V), then, if asked for, the decayed column sums.
  *   K, V    dev [batch][n_kv_heads][T][head_dim];  Q dev [batch][n_q_heads][T][head_dim];
  *           storage dtype of the cache (fp16 or bf16; ZSM_ERR_UNSUPPORTED for fp32), 16-byte aligned
  *   out     dev [batch][n_q_heads][T][head_dim], storage dtype, written
