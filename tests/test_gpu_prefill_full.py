@@ -234,6 +234,45 @@ def test_prefill_attention_long_prompt(zb):
         cache.close()
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_prefill_attention_rising_maximum(zb, dtype):
+    """Logits that keep growing with the key position, by about 18 in the log2 domain per key
+    tile, for the odd query rows only: the reference maximum of those rows moves at every tile, so
+    their rows of the output accumulator are rescaled in tensor memory again and again, while the
+    even rows of the same warps (flat logits) keep theirs.  Output against SDPA in fp64, log-sum-exp
+    against torch.logsumexp."""
+    T, d, G = 700, 128, 2
+    w = wl.Workload("attnrise", 1, 1, 2 * G, 2, d, dtype, T, 0, T, None, 44)
+    cache = GpuCache(zb, w, [[4, 4]], [[6, 6]], [[1, 1]])
+    try:
+        K, V, Q = wl.prompt(w, 0)
+        ramp = torch.arange(T, dtype=torch.float32) * 0.1      # logit gain per key position
+        K = K.float() * 0.05
+        K[..., 0] = ramp                                        # keys grow along the first axis
+        Q = Q.float() * 0.05
+        Q[..., 0] = 0.0
+        Q[:, :, 1::2, 0] = float(np.sqrt(d))                    # odd rows: logit = 0.1 * position
+        K, Q = K.to(w.torch_dtype), Q.to(w.torch_dtype)
+        out = torch.full((1, 2 * G, T, d), float("nan"), dtype=w.torch_dtype, device="cuda")
+        lse = torch.full((1, 2 * G, T), float("nan"), dtype=torch.float32, device="cuda")
+        zb.zsm_prefill_attention(cache.h, K.cuda(), V.cuda(), Q.cuda(), T, out, lse)
+        torch.cuda.synchronize()
+        assert cache.status() == 0
+        Kd = K.double().repeat_interleave(G, dim=1)
+        Vd = V.double().repeat_interleave(G, dim=1)
+        Qd = Q.double()
+        ref = torch.nn.functional.scaled_dot_product_attention(Qd, Kd, Vd, is_causal=True)
+        torch.testing.assert_close(out.cpu().double(), ref, atol=2e-3, rtol=1e-2)
+        logits = torch.einsum("bhqd,bhkd->bhqk", Qd, Kd) / np.sqrt(float(d))
+        mask = torch.tril(torch.ones(T, T, dtype=torch.bool))
+        ref_lse = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
+        # the rise over the prompt is what the test is about: 0.1 * 699 nats on the odd rows
+        assert float(ref_lse[0, 0, T - 1]) > 60.0 and abs(float(ref_lse[0, 0, T - 2])) < 10.0
+        torch.testing.assert_close(lse.cpu().double(), ref_lse, atol=1e-4, rtol=1e-5)
+    finally:
+        cache.close()
+
+
 def test_prefill_attention_argument_errors(zb):
     w = wl.Workload("attnerr", 1, 1, 2, 2, 64, "f32", 32, 0, 32, None, 43)
     cache = GpuCache(zb, w, [[4, 4]], [[4, 4]], [[1, 1]])
