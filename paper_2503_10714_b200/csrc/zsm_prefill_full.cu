@@ -899,6 +899,204 @@ __global__ void __launch_bounds__(kAoThreads, 1)
                      : "memory");
 }
 
+// ---------------------------------------------------------------------------
+// Window scoring of the prompt pass (App. B: the last W prompt queries score the keys) on tcgen05:
+// the scaled, causally masked logits of a unit's G*W window queries against every key, fp32
+// [G*W][T], and per 128-key chunk each query row's (max, sum exp) -- the same outputs as the
+// warp-level kernel of the prompt pass, for windows of G*W = 32, 64, 96 or 128 rows.
+// Persistent CTAs, grid (CTAs per unit, units): CTA x takes the unit's chunks x, x + gridDim.x, ...
+// The window's queries are resident in shared memory (one TMA box of G*W rows); 128-key chunks
+// stream through a two-stage ring (TMA, 128-byte swizzle).  One thread requests chunks and issues
+// the products: positions are the M side (a chunk's 128 keys = the 128 tensor-memory lanes), the
+// window's rows the N side, two accumulators of G*W columns so the next chunk's product runs under
+// this chunk's write-out.  Write-out, 32 query rows at a time: four warps move their lanes'
+// columns into a shared tile [row][position]; then all eight warps take four rows each -- a lane
+// handles positions lane, lane + 32, ... -- which gives coalesced row writes and the row's
+// (max, sum exp) of the chunk by warp shuffles.  Two CTAs share an SM.
+// ---------------------------------------------------------------------------
+constexpr int kWlThreads = 288;  // 8 write-out warps + the warp that requests and issues
+constexpr int kWlStages = 2;
+constexpr int kWlLT = kTcRows + 4;  // padded row of the shared tile (floats)
+enum : int32_t { WW_Q = 61, WW_K = 62, WW_ACC = 63, WW_MMA = 64 };
+
+template <int D>
+struct WlSmem {
+    static constexpr int KB = D / kTcKBlock;
+    static constexpr int KBLOCK = kTcRows * 128;
+    static constexpr int TILE = KB * KBLOCK;  // a chunk of keys
+    static constexpr int k = 0;
+    static constexpr int q = kWlStages * TILE;  // up to 128 query rows
+    static int lt(int GW) { return q + KB * GW * 128; }
+    static int bars(int GW) { return lt(GW) + 32 * kWlLT * 4; }
+    static int total(int GW) { return bars(GW) + 128 + 1024; }
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kWlThreads, 2)
+    window_logits_tc_kernel(const WindowLogitsParams p, const __grid_constant__ CUtensorMap map_k,
+                            const __grid_constant__ CUtensorMap map_q) {
+    using L = WlSmem<D>;
+    constexpr int KS = D / 16;
+    constexpr int CH = kTcRows;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const int GW = p.G * p.W;
+    float *lt = reinterpret_cast<float *>(smem + L::lt(GW));
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + L::bars(GW));  // [2] chunk landed
+    uint64_t *mma_bar = full_bar + kWlStages;                               // [2] product finished
+    uint64_t *acc_free = mma_bar + 2;                                       // [2] accumulator read
+    uint64_t *q_bar = acc_free + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_bar + 1);
+    volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(tmem_slot + 2);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ul = blockIdx.y;
+    const int b = ul / p.n_kv_heads, h = ul % p.n_kv_heads;
+    const int T_len = p.T, W = p.W;
+    const int n_chunks = (T_len + CH - 1) / CH;
+    const int n_my = blockIdx.x < n_chunks ? (n_chunks - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+    // tensor-memory columns: two accumulators of GW columns, rounded up to a power of two
+    const uint32_t tmem_cols = GW <= 32 ? 64u : (GW <= 64 ? 128u : 256u);
+
+    if (tid == 0) {
+        for (int s = 0; s < kWlStages; ++s) mbar_init(&full_bar[s], 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&mma_bar[s], 1);
+            mbar_init(&acc_free[s], 4);
+        }
+        mbar_init(q_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(tmem_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool ok = true;
+
+    if (warp == 8) {
+        if (lane == 0 && n_my > 0) {
+            auto load_chunk = [&](int i) {  // this CTA's i-th chunk into stage i % 2
+                const int s = i % kWlStages;
+                const int c = blockIdx.x + i * gridDim.x;
+                mbar_arrive_expect_tx(&full_bar[s], L::TILE);
+#pragma unroll
+                for (int kb = 0; kb < L::KB; ++kb)
+                    tma_load_3d(smem + L::k + s * L::TILE + kb * L::KBLOCK, &map_k, kb * kTcKBlock, c * CH, ul,
+                                &full_bar[s]);
+            };
+            // the unit's window: rows (b, h G .. h G + G - 1, 0 .. W - 1) are consecutive
+            mbar_arrive_expect_tx(q_bar, L::KB * GW * 128);
+#pragma unroll
+            for (int kb = 0; kb < L::KB; ++kb)
+                tma_load_3d(smem + L::q + kb * GW * 128, &map_q, kb * kTcKBlock,
+                            (b * p.n_kv_heads + h) * GW, 0, q_bar);
+            for (int i = 0; i < kWlStages && i < n_my; ++i) load_chunk(i);
+            const uint32_t f = Elem<T>::kIsBf16 ? 1u : 0u;
+            const uint32_t idesc = (1u << 4) | (f << 7) | (f << 10) | ((static_cast<uint32_t>(GW) >> 3) << 17) |
+                                   ((kTcRows >> 4) << 24);
+            ok = mbar_wait_bounded(q_bar, 0, abort_flag, p.status, WW_Q);
+            for (int i = 0; i < n_my && ok; ++i) {
+                const int s = i % kWlStages, buf = i & 1;
+                ok = mbar_wait_bounded(&full_bar[s], (i / kWlStages) & 1u, abort_flag, p.status, WW_K);
+                if (ok && i >= 2)
+                    ok = mbar_wait_bounded(&acc_free[buf], ((i - 2) >> 1) & 1u, abort_flag, p.status, WW_ACC);
+                if (!ok) break;
+                tc_fence_after();
+                const uint8_t *kt = smem + L::k + s * L::TILE;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int ko = (ks / 4) * L::KBLOCK + (ks % 4) * 32;   // 16 elements = 32 bytes on
+                    const int qo = (ks / 4) * GW * 128 + (ks % 4) * 32;
+                    umma_f16_ss(tmem_base + buf * GW, umma_desc_sw128(kt + ko), umma_desc_sw128(smem + L::q + qo),
+                                idesc, ks > 0);
+                }
+                umma_commit(&mma_bar[buf]);
+                // the finished product frees the chunk's stage: request the chunk two on
+                if (i + kWlStages < n_my) {
+                    ok = mbar_wait_bounded(&mma_bar[buf], (i >> 1) & 1u, abort_flag, p.status, WW_MMA);
+                    if (ok) load_chunk(i + kWlStages);
+                }
+            }
+            if (!ok) {
+                // copies that were requested may still land: give them time before the memory goes away
+                const uint64_t t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    } else {
+        float *logits = p.logits + (size_t)ul * GW * T_len;
+        float2 *partial = p.partial + (size_t)ul * GW * n_chunks;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        for (int i = 0; i < n_my && ok; ++i) {
+            const int buf = i & 1;
+            const int chunk = blockIdx.x + i * gridDim.x;
+            const int t0 = chunk * CH;
+            // a wait gives the same answer to every thread that asks for the same phase, so the
+            // eight warps leave the loop at the same chunk and none is left at the named barrier
+            if (!mbar_wait_bounded(&mma_bar[buf], (i >> 1) & 1u, abort_flag, p.status, WW_MMA)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            for (int qb = 0; qb < GW; qb += 32) {
+                if (warp < 4) {
+                    // lanes = positions 32 warp .. of the chunk, columns = query rows qb .. qb + 31
+                    uint32_t v[32];
+                    tmem_ld32(lane_base + buf * GW + qb, v);
+                    if (qb + 32 >= GW) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&acc_free[buf]);  // this warp is done with the accumulator
+                    }
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) lt[c * kWlLT + warp * 32 + lane] = __uint_as_float(v[c]) * p.scale;
+                }
+                named_bar_sync(1, 256);
+                // warp w: query rows 4w .. 4w+3 of the block; lane: positions lane + 32 i
+#pragma unroll
+                for (int jr = 0; jr < 4; ++jr) {
+                    const int gw = qb + warp * 4 + jr;
+                    const int tau = T_len - W + (gw % W);  // the query's own position: keys 0..tau
+                    float m = -INFINITY;
+                    float lg[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int t = t0 + lane + 32 * k;
+                        lg[k] = (t < T_len && t <= tau) ? lt[(warp * 4 + jr) * kWlLT + lane + 32 * k] : -INFINITY;
+                        if (t < T_len) logits[(size_t)gw * T_len + t] = lg[k];
+                        m = fmaxf(m, lg[k]);
+                    }
+#pragma unroll
+                    for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                    float sum = 0.f;
+                    if (m > -INFINITY) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) sum += expf(lg[k] - m);
+                    }
+#pragma unroll
+                    for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                    if (lane == 0) partial[(size_t)gw * n_chunks + chunk] = make_float2(m, sum);
+                }
+                named_bar_sync(1, 256);  // the tile is rewritten by the next block of rows
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
+                     : "memory");
+}
+
 // cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link
 // against the driver library directly.
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -931,6 +1129,38 @@ bool make_map(CUtensorMap *map, const void *base, int heads, int T, int D, bool 
               const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// [rows][D] row-major, 16-bit elements, seen as (d, row, 1): boxes of 64 x box_rows with the
+// 128-byte swizzle.
+bool make_map_rows(CUtensorMap *map, const void *base, size_t rows, int D, int box_rows, bool bf16) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t gdim[3] = {(cuuint64_t)D, (cuuint64_t)rows, 1};
+    const cuuint64_t gstride[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kTcKBlock, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+              const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename T, int D>
+int launch_window_one(const WindowLogitsParams &p, int grid_x, cudaStream_t stream) {
+    const int GW = p.G * p.W;
+    CUtensorMap map_k, map_q;
+    if (!make_map(&map_k, p.K, p.units, p.T, D, Elem<T>::kIsBf16) ||
+        !make_map_rows(&map_q, p.Qw, (size_t)p.units * GW, D, GW, Elem<T>::kIsBf16))
+        return static_cast<int>(cudaErrorInvalidValue);
+    window_logits_tc_kernel<T, D><<<dim3(grid_x, p.units), kWlThreads, WlSmem<D>::total(GW), stream>>>(p, map_k, map_q);
+    return static_cast<int>(cudaGetLastError());
+}
+
+template <typename T, int D>
+int prepare_window_one() {
+    return static_cast<int>(cudaFuncSetAttribute(window_logits_tc_kernel<T, D>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, WlSmem<D>::total(128)));
 }
 
 template <typename T, int D>
@@ -1023,12 +1253,29 @@ int launch_full_scores(int dtype, int D, const FullScoreParams &p, cudaStream_t 
     return -1;
 }
 
+bool window_logits_tc_supported(int GW) { return GW >= 32 && GW <= 128 && GW % 32 == 0; }
+
+int launch_window_logits_tc(int dtype, int D, const WindowLogitsParams &p, int grid_x, cudaStream_t stream) {
+    if (!window_logits_tc_supported(p.G * p.W)) return -1;
+    if (dtype == 1 && D == 64) return launch_window_one<__half, 64>(p, grid_x, stream);
+    if (dtype == 1 && D == 128) return launch_window_one<__half, 128>(p, grid_x, stream);
+    if (dtype == 2 && D == 64) return launch_window_one<__nv_bfloat16, 64>(p, grid_x, stream);
+    if (dtype == 2 && D == 128) return launch_window_one<__nv_bfloat16, 128>(p, grid_x, stream);
+    return -1;
+}
+
 int prepare_full_scores(int dtype, int D) {
     int rc = -1;
-    if (dtype == 1 && D == 64) rc = prepare_full_one<__half, 64>() | prepare_attn_one<__half, 64>();
-    if (dtype == 1 && D == 128) rc = prepare_full_one<__half, 128>() | prepare_attn_one<__half, 128>();
-    if (dtype == 2 && D == 64) rc = prepare_full_one<__nv_bfloat16, 64>() | prepare_attn_one<__nv_bfloat16, 64>();
-    if (dtype == 2 && D == 128) rc = prepare_full_one<__nv_bfloat16, 128>() | prepare_attn_one<__nv_bfloat16, 128>();
+    if (dtype == 1 && D == 64)
+        rc = prepare_full_one<__half, 64>() | prepare_attn_one<__half, 64>() | prepare_window_one<__half, 64>();
+    if (dtype == 1 && D == 128)
+        rc = prepare_full_one<__half, 128>() | prepare_attn_one<__half, 128>() | prepare_window_one<__half, 128>();
+    if (dtype == 2 && D == 64)
+        rc = prepare_full_one<__nv_bfloat16, 64>() | prepare_attn_one<__nv_bfloat16, 64>() |
+             prepare_window_one<__nv_bfloat16, 64>();
+    if (dtype == 2 && D == 128)
+        rc = prepare_full_one<__nv_bfloat16, 128>() | prepare_attn_one<__nv_bfloat16, 128>() |
+             prepare_window_one<__nv_bfloat16, 128>();
     return rc;
 }
 

@@ -27,6 +27,19 @@ int launch_row_statistics(int dtype, int D, const FullScoreParams &p, cudaStream
 // every query row's log-sum-exp into p.lse_out (required; p.lse is not read); V [batch][n_kv_heads][T][d].
 int launch_attention_output(int dtype, int D, const FullScoreParams &p, const void *V, void *out,
                             cudaStream_t stream);
+// Window scoring of the prompt pass on tcgen05 (16-bit storage, windows of G*W = 32, 64, 96, 128 rows).
+struct WindowLogitsParams {
+    const void *K;     // [units][T][d]
+    const void *Qw;    // [batch][n_q_heads][W][d]: a unit's G*W rows are consecutive
+    float *logits;     // fp32 [units][G*W][T], scaled, causally masked (-inf)
+    float2 *partial;   // [units][G*W][chunks of 128 keys]: (max, sum exp) of the chunk
+    int32_t *status;
+    int32_t units, n_kv_heads, T, W, G;
+    float scale;
+};
+bool window_logits_tc_supported(int GW);
+// grid_x persistent CTAs per unit.  Returns a cudaError_t as int; -1: no kernel for this case.
+int launch_window_logits_tc(int dtype, int D, const WindowLogitsParams &p, int grid_x, cudaStream_t stream);
 // Raises the kernels' dynamic shared-memory limit; returns a cudaError_t as int (-1: no kernel).
 int prepare_full_scores(int dtype, int D);
 
