@@ -14,6 +14,7 @@
 //                          the row-per-warp form holds the merged rows in registers (B_r <= 128)
 //   P5  prefill_gather     survivors' rows, scores and positions into the unit's slots
 #include "zsm_prefill.cuh"
+#include "zsm_prefill_full.cuh"
 
 #include <algorithm>
 
@@ -1321,7 +1322,28 @@ int launch_all(const PrefillParams &p, int max_br, cudaStream_t stream) {
             // at most two CTAs per SM over the whole launch -- one wave -- each walking its share
             // of a unit's chunks
             const int per_unit = std::max(1, std::min(n_chunks, (2 * p.n_sm) / p.units));
-            prefill_logits_mma_kernel<T, D><<<dim3(per_unit, p.units), kP1Threads, logits_mma_smem_bytes<D>(), stream>>>(p);
+            const int GW = p.G * p.W;
+            if (window_logits_tc_supported(GW)) {
+                // windows of 32 .. 128 query rows: the tcgen05 form
+                WindowLogitsParams wp;
+                wp.K = p.K;
+                wp.Qw = p.Qw;
+                wp.logits = reinterpret_cast<float *>(p.ws + p.wl.logits);
+                wp.partial = reinterpret_cast<float2 *>(p.ws + p.wl.partial);
+                wp.status = p.status;
+                wp.units = p.units;
+                wp.n_kv_heads = p.n_kv_heads;
+                wp.T = p.T;
+                wp.W = p.W;
+                wp.G = p.G;
+                wp.scale = p.scale;
+                // two CTAs fit an SM up to 64 rows, one beyond (the window's rows are resident)
+                const int ctas = GW <= 64 ? 2 * p.n_sm : p.n_sm;
+                const int px = std::max(1, std::min(n_chunks, ctas / p.units));
+                const int rc = launch_window_logits_tc(Elem<T>::kIsBf16 ? 2 : 1, D, wp, px, stream);
+                if (rc != 0) return rc;
+            } else
+                prefill_logits_mma_kernel<T, D><<<dim3(per_unit, p.units), kP1Threads, logits_mma_smem_bytes<D>(), stream>>>(p);
         }
         else
             prefill_logits_kernel<T, D><<<dim3(n_chunks, p.units), 256, sm, stream>>>(p);

@@ -926,9 +926,9 @@ struct WlSmem {
     static constexpr int TILE = KB * KBLOCK;  // a chunk of keys
     static constexpr int k = 0;
     static constexpr int q = kWlStages * TILE;  // up to 128 query rows
-    static int lt(int GW) { return q + KB * GW * 128; }
-    static int bars(int GW) { return lt(GW) + 32 * kWlLT * 4; }
-    static int total(int GW) { return bars(GW) + 128 + 1024; }
+    static __host__ __device__ constexpr int lt(int GW) { return q + KB * GW * 128; }
+    static __host__ __device__ constexpr int bars(int GW) { return lt(GW) + 32 * kWlLT * 4; }
+    static __host__ __device__ constexpr int total(int GW) { return bars(GW) + 128 + 1024; }
 };
 
 template <typename T, int D>

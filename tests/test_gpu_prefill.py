@@ -55,6 +55,28 @@ def test_prompt_pass_all_kernel_variants(zb, oracle, dtype, head_dim, group):
     assert stats.selections > 4000 and stats.merges > 3500
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("head_dim,group,window", [(128, 1, 32), (64, 2, 32), (128, 4, 24), (128, 4, 32),
+                                                   (64, 1, 64)])
+def test_prompt_pass_window_scoring_on_tcgen05(zb, oracle, dtype, head_dim, group, window):
+    """Windows of G * W = 32, 64, 96 and 128 query rows take the tcgen05 form of the window
+    scoring (one, two, three and four blocks of 32 rows per chunk; both accumulators, both chunk
+    stages and every barrier phase wrap: 11 chunks over at most 3 CTAs per unit here); the prompt
+    ends inside a chunk.  Scores, selection, merge targets and state against the oracle."""
+    w = wl.Workload("pptc", 1, 2, 2 * group, 2, head_dim, dtype, 1333, 0, window, None, 45)
+    bp = np.array([[16, 40]])
+    bc = np.array([[20, 61]])
+    br = np.array([[2, 5]])
+    cache = GpuCache(zb, w, bp, bc, br)
+    stats = ParityStats()
+    try:
+        prefill_all_units(zb, oracle, w, cache, 0, stats)
+        assert cache.status() == 0
+    finally:
+        cache.close()
+    assert stats.selections > 4000
+
+
 @pytest.mark.parametrize("T,window", [(5, 5), (30, 8), (48, 48), (129, 1), (300, 300)])
 def test_prompt_lengths_around_the_budgets(zb, oracle, T, window):
     """Prompts shorter than B_p, shorter than B_p + B_c (nothing evicted), barely longer
