@@ -1036,34 +1036,33 @@ __global__ void __launch_bounds__(kWlThreads, 2)
         float *logits = p.logits + (size_t)ul * GW * T_len;
         float2 *partial = p.partial + (size_t)ul * GW * n_chunks;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        for (int i = 0; i < n_my && ok; ++i) {
+        for (int i = 0; i < n_my; ++i) {
             const int buf = i & 1;
             const int chunk = blockIdx.x + i * gridDim.x;
             const int t0 = chunk * CH;
-            // a wait gives the same answer to every thread that asks for the same phase, so the
-            // eight warps leave the loop at the same chunk and none is left at the named barrier
-            if (!mbar_wait_bounded(&mma_bar[buf], (i >> 1) & 1u, abort_flag, p.status, WW_MMA)) {
-                ok = false;
-                break;
-            }
+            // A warp whose wait gave up does no more work and no more waiting, but it still walks
+            // the named barriers below (they have no time limit), so no other warp is left there.
+            if (ok && !mbar_wait_bounded(&mma_bar[buf], (i >> 1) & 1u, abort_flag, p.status, WW_MMA)) ok = false;
             tc_fence_after();
             for (int qb = 0; qb < GW; qb += 32) {
-                if (warp < 4) {
+                if (ok && warp < 4) {
                     // lanes = positions 32 warp .. of the chunk, columns = query rows qb .. qb + 31
                     uint32_t v[32];
                     tmem_ld32(lane_base + buf * GW + qb, v);
-                    if (qb + 32 >= GW) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&acc_free[buf]);  // this warp is done with the accumulator
-                    }
+                    tc_fence_before();
 #pragma unroll
                     for (int c = 0; c < 32; ++c) lt[c * kWlLT + warp * 32 + lane] = __uint_as_float(v[c]) * p.scale;
                 }
                 named_bar_sync(1, 256);
+                // The accumulator goes back only now, behind a barrier of all eight warps: every
+                // warp has then passed its wait for this chunk's product.  Handed back by the four
+                // loading warps alone, the barrier of that wait could complete twice more -- the
+                // next product but one needs nothing else -- before a late warp has looked at it,
+                // and that warp would wait for a phase that can no longer come.
+                if (qb + 32 >= GW && warp < 4 && lane == 0) mbar_arrive(&acc_free[buf]);
                 // warp w: query rows 4w .. 4w+3 of the block; lane: positions lane + 32 i
 #pragma unroll
-                for (int jr = 0; jr < 4; ++jr) {
+                for (int jr = 0; jr < 4 && ok; ++jr) {
                     const int gw = qb + warp * 4 + jr;
                     const int tau = T_len - W + (gw % W);  // the query's own position: keys 0..tau
                     float m = -INFINITY;
