@@ -130,6 +130,51 @@ def test_layer_with_more_units_than_resident_ctas(zb, oracle):
         cache.close()
 
 
+def test_prompt_passes_on_four_streams_repeat_the_serial_result(zb):
+    """Eight layers' prompt passes round-robin on four streams, three times over, against the
+    same layers compressed one after another: scores, eviction flags and merge targets must be
+    bit-identical (every kernel of the pass is deterministic).  The window scoring kernel's
+    write-out warps run at uneven pace when launches of several streams share the SMs."""
+    w = wl.Workload("four", 8, 1, 8, 8, 128, "f16", 6000, 0, 32, None, 46)
+    bp, bc, br = np.full((8, 8), 40), np.full((8, 8), 60), np.full((8, 8), 4)
+    cache = GpuCache(zb, w, bp, bc, br)
+    try:
+        T = w.prompt_len
+        dev = [[t.cuda() for t in wl.prompt(w, layer)] for layer in range(w.n_layers)]
+
+        def outputs():
+            return {"scores": torch.empty(w.batch, w.n_kv_heads, T, dtype=torch.float32, device="cuda"),
+                    "evicted": torch.zeros(w.batch, w.n_kv_heads, T, dtype=torch.uint8, device="cuda"),
+                    "targets": torch.full((w.batch, w.n_kv_heads, T), -9, dtype=torch.int32, device="cuda")}
+
+        need = zb.zsm_prefill_workspace_bytes(cache.h, T, w.window)
+        wss = [torch.empty(need, dtype=torch.uint8, device="cuda") for _ in range(4)]
+        serial = []
+        for layer in range(w.n_layers):
+            d = outputs()
+            K, V, Qw = dev[layer]
+            zb.zsm_prefill_compress(cache.h, layer, K, V, Qw, None, T, w.window, wss[0], d["scores"],
+                                    d["evicted"], d["targets"])
+            serial.append(d)
+        torch.cuda.synchronize()
+        streams = [torch.cuda.Stream() for _ in range(4)]
+        for rep in range(3):
+            side = []
+            for layer in range(w.n_layers):
+                d = outputs()
+                K, V, Qw = dev[layer]
+                zb.zsm_prefill_compress(cache.h, layer, K, V, Qw, None, T, w.window, wss[layer % 4],
+                                        d["scores"], d["evicted"], d["targets"], stream=streams[layer % 4])
+                side.append(d)
+            torch.cuda.synchronize()
+            assert cache.status() == 0
+            for layer in range(w.n_layers):
+                for key in ("scores", "evicted", "targets"):
+                    assert torch.equal(side[layer][key], serial[layer][key]), (rep, layer, key)
+    finally:
+        cache.close()
+
+
 def test_layers_compressed_side_by_side_on_two_streams(zb, oracle):
     """Layers are independent: their prompt passes may run at the same time on different
     streams, each with a workspace of its own.  Three layers on two streams (the third queues
