@@ -127,6 +127,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Eight columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Sixteen columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -948,12 +969,14 @@ __global__ void __launch_bounds__(kAoThreads, 1)
 // stream through a two-stage ring (TMA, 128-byte swizzle).  One thread requests chunks and issues
 // the products: positions are the M side (a chunk's 128 keys = the 128 tensor-memory lanes), the
 // window's rows the N side, two accumulators of G*W columns so the next chunk's product runs under
-// this chunk's write-out.  Write-out, 32 query rows at a time: four warps move their lanes'
-// columns into a shared tile [row][position]; then all eight warps take four rows each -- a lane
+// this chunk's write-out.  Write-out, 32 query rows at a time: the NW warps move their lanes'
+// columns (128 / NW each) into a shared tile [row][position], then take 32 / NW rows each -- a lane
 // handles positions lane, lane + 32, ... -- which gives coalesced row writes and the row's
-// (max, sum exp) of the chunk by warp shuffles.  Two CTAs share an SM.
+// (max, sum exp) of the chunk by warp shuffles; two tiles taken in turn, one named barrier per
+// round.  Two CTAs share an SM for windows of up to 64 rows.
 // ---------------------------------------------------------------------------
-constexpr int kWlThreads = 288;  // 8 write-out warps + the warp that requests and issues
+// NW write-out warps (8 for windows of up to 64 rows, where two CTAs share an SM; 16 beyond, where the
+// CTA has the SM to itself) + the warp that requests and issues
 constexpr int kWlStages = 2;
 constexpr int kWlLT = kTcRows + 4;  // padded row of the shared tile (floats)
 enum : int32_t { WW_Q = 61, WW_K = 62, WW_ACC = 63, WW_MMA = 64 };
@@ -966,12 +989,12 @@ struct WlSmem {
     static constexpr int k = 0;
     static constexpr int q = kWlStages * TILE;  // up to 128 query rows
     static __host__ __device__ constexpr int lt(int GW) { return q + KB * GW * 128; }
-    static __host__ __device__ constexpr int bars(int GW) { return lt(GW) + 32 * kWlLT * 4; }
+    static __host__ __device__ constexpr int bars(int GW) { return lt(GW) + 2 * 32 * kWlLT * 4; }  // two tiles
     static __host__ __device__ constexpr int total(int GW) { return bars(GW) + 128 + 1024; }
 };
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kWlThreads, 2)
+template <typename T, int D, int NW>
+__global__ void __launch_bounds__(NW * 32 + 32, NW == 8 ? 2 : 1)
     window_logits_tc_kernel(const WindowLogitsParams p, const __grid_constant__ CUtensorMap map_k,
                             const __grid_constant__ CUtensorMap map_q) {
     using L = WlSmem<D>;
@@ -1021,7 +1044,7 @@ __global__ void __launch_bounds__(kWlThreads, 2)
     const uint32_t tmem_base = *tmem_slot;
     bool ok = true;
 
-    if (warp == 8) {
+    if (warp == NW) {
         if (lane == 0 && n_my > 0) {
             auto load_chunk = [&](int i) {  // this CTA's i-th chunk into stage i % 2
                 const int s = i % kWlStages;
@@ -1075,6 +1098,7 @@ __global__ void __launch_bounds__(kWlThreads, 2)
         float *logits = p.logits + (size_t)ul * GW * T_len;
         float2 *partial = p.partial + (size_t)ul * GW * n_chunks;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        int rounds = 0;
         for (int i = 0; i < n_my; ++i) {
             const int buf = i & 1;
             const int chunk = blockIdx.x + i * gridDim.x;
@@ -1084,32 +1108,44 @@ __global__ void __launch_bounds__(kWlThreads, 2)
             if (ok && !mbar_wait_bounded(&mma_bar[buf], (i >> 1) & 1u, abort_flag, p.status, WW_MMA)) ok = false;
             tc_fence_after();
             for (int qb = 0; qb < GW; qb += 32) {
-                if (ok && warp < 4) {
-                    // lanes = positions 32 warp .. of the chunk, columns = query rows qb .. qb + 31
-                    uint32_t v[32];
-                    tmem_ld32(lane_base + buf * GW + qb, v);
+                // two tiles taken in turn: a round's barrier also says that every warp is done
+                // with the rows of the round before, so the tile of the round before that is free
+                float *tile = lt + (rounds & 1) * 32 * kWlLT;
+                ++rounds;
+                if (ok) {
+                    // lanes = positions 32 (warp % 4) .. of the chunk; warp w takes the query rows
+                    // qb + CW (w / 4) .. of the block
+                    constexpr int CW = 128 / NW;  // columns per warp: 16 or 8
+                    uint32_t v[CW];
+                    const int c0 = (warp >> 2) * CW;
+                    if constexpr (CW == 16)
+                        tmem_ld16(lane_base + buf * GW + qb + c0, v);
+                    else
+                        tmem_ld8(lane_base + buf * GW + qb + c0, v);
                     tc_fence_before();
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) lt[c * kWlLT + warp * 32 + lane] = __uint_as_float(v[c]) * p.scale;
+                    for (int c = 0; c < CW; ++c)
+                        tile[(c0 + c) * kWlLT + (warp & 3) * 32 + lane] = __uint_as_float(v[c]) * p.scale;
                 }
-                named_bar_sync(1, 256);
-                // The accumulator goes back only now, behind a barrier of all eight warps: every
-                // warp has then passed its wait for this chunk's product.  Handed back by the four
-                // loading warps alone, the barrier of that wait could complete twice more -- the
-                // next product but one needs nothing else -- before a late warp has looked at it,
-                // and that warp would wait for a phase that can no longer come.
+                named_bar_sync(1, NW * 32);
+                // The accumulator goes back only now, behind a barrier of all write-out warps: every
+                // warp has then passed its wait for this chunk's product.  Handed back by the
+                // loading warps as they finish, the barrier of that wait could complete twice more
+                // -- the next product but one needs nothing else -- before a late warp has looked
+                // at it, and that warp would wait for a phase that can no longer come.
                 if (qb + 32 >= GW && warp < 4 && lane == 0) mbar_arrive(&acc_free[buf]);
-                // warp w: query rows 4w .. 4w+3 of the block; lane: positions lane + 32 i
+                // warp w: query rows RW w .. of the block (RW = 4 or 2); lane: positions lane + 32 i
+                constexpr int RW = 32 / NW;
 #pragma unroll
-                for (int jr = 0; jr < 4 && ok; ++jr) {
-                    const int gw = qb + warp * 4 + jr;
+                for (int jr = 0; jr < RW && ok; ++jr) {
+                    const int gw = qb + warp * RW + jr;
                     const int tau = T_len - W + (gw % W);  // the query's own position: keys 0..tau
                     float m = -INFINITY;
                     float lg[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const int t = t0 + lane + 32 * k;
-                        lg[k] = (t < T_len && t <= tau) ? lt[(warp * 4 + jr) * kWlLT + lane + 32 * k] : -INFINITY;
+                        lg[k] = (t < T_len && t <= tau) ? tile[(warp * RW + jr) * kWlLT + lane + 32 * k] : -INFINITY;
                         if (t < T_len) logits[(size_t)gw * T_len + t] = lg[k];
                         m = fmaxf(m, lg[k]);
                     }
@@ -1124,7 +1160,6 @@ __global__ void __launch_bounds__(kWlThreads, 2)
                     for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
                     if (lane == 0) partial[(size_t)gw * n_chunks + chunk] = make_float2(m, sum);
                 }
-                named_bar_sync(1, 256);  // the tile is rewritten by the next block of rows
             }
         }
     }
@@ -1191,14 +1226,21 @@ int launch_window_one(const WindowLogitsParams &p, int grid_x, cudaStream_t stre
     if (!make_map(&map_k, p.K, p.units, p.T, D, Elem<T>::kIsBf16) ||
         !make_map_rows(&map_q, p.Qw, (size_t)p.units * GW, D, GW, Elem<T>::kIsBf16))
         return static_cast<int>(cudaErrorInvalidValue);
-    window_logits_tc_kernel<T, D><<<dim3(grid_x, p.units), kWlThreads, WlSmem<D>::total(GW), stream>>>(p, map_k, map_q);
+    if (GW <= 64)
+        window_logits_tc_kernel<T, D, 8><<<dim3(grid_x, p.units), 8 * 32 + 32, WlSmem<D>::total(GW), stream>>>(p, map_k, map_q);
+    else
+        window_logits_tc_kernel<T, D, 16><<<dim3(grid_x, p.units), 16 * 32 + 32, WlSmem<D>::total(GW), stream>>>(p, map_k, map_q);
     return static_cast<int>(cudaGetLastError());
 }
 
 template <typename T, int D>
 int prepare_window_one() {
-    return static_cast<int>(cudaFuncSetAttribute(window_logits_tc_kernel<T, D>,
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, WlSmem<D>::total(128)));
+    cudaError_t e = cudaFuncSetAttribute(window_logits_tc_kernel<T, D, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         WlSmem<D>::total(64));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(window_logits_tc_kernel<T, D, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 WlSmem<D>::total(128));
+    return static_cast<int>(e);
 }
 
 template <typename T, int D>
