@@ -882,7 +882,7 @@ __global__ void __launch_bounds__(kAoThreads, 1)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t w[16];                  // 32 weights, packed in pairs
-                    uint32_t wl[kSplitW ? 16 : 1];   // their remainders
+                    [[maybe_unused]] uint32_t wl[kSplitW ? 16 : 1];   // their remainders
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
                         float x0, x1;
