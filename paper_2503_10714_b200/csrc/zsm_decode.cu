@@ -921,6 +921,13 @@ __global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 
             }
             release();
         }
+        // The partial outputs are folded through the memory the weights occupy: keep the new
+        // token's weights (the last entries) in registers, and let every warp finish reading
+        // weights before the first partial is written.
+        float pnew[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) pnew[g] = probs[(n_ent - 1) * G + g];
+        csync();
         // fold the RPW row groups of a warp, then the warps
 #pragma unroll
         for (int g = 0; g < G; ++g) {
@@ -951,12 +958,14 @@ __global__ void __launch_bounds__(WIDE ? kMaxThreads : kPairThreads, WIDE ? 1 : 
         {
             const T *vn = reinterpret_cast<const T *>(vn_raw);
             T *out = static_cast<T *>(p.out) + (size_t)ul * G * D;
-            for (int k = tid; k < G * D; k += NT) {
-                const int g = k / D, dim = k % D;
-                float sum = 0.f;
-                for (int wv = 0; wv < NW; ++wv) sum += opart[(wv * G + g) * D + dim];
-                sum = fmaf(probs[(n_ent - 1) * G + g], E::to_float(vn[dim]), sum);
-                out[k] = E::from_float(sum * inv[g]);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                for (int dim = tid; dim < D; dim += NT) {
+                    float sum = 0.f;
+                    for (int wv = 0; wv < NW; ++wv) sum += opart[(wv * G + g) * D + dim];
+                    sum = fmaf(pnew[g], E::to_float(vn[dim]), sum);
+                    out[g * D + dim] = E::from_float(sum * inv[g]);
+                }
             }
         }
         csync();  // shared scratch is free for the next unit

@@ -57,11 +57,15 @@ __host__ __device__ inline DecodeSmem decode_smem_layout(int stages, int G, int 
     L.ring = take(static_cast<uint32_t>(stages) * kTileBytes);
     L.bars = take((2u * static_cast<uint32_t>(stages) + 6u) * 8u);
     L.flags = take(64u);
-    L.probs = take(static_cast<uint32_t>(G) * l_stride * 4u);
+    // the warps' partial outputs are folded where the weights were (the weights are dead once the
+    // output pass is over): one region, sized for the larger of the two
+    const uint32_t probs_bytes = static_cast<uint32_t>(G) * l_stride * 4u;
+    const uint32_t opart_bytes = static_cast<uint32_t>(consumer_warps) * G * D * 4u;
+    L.probs = take(probs_bytes > opart_bytes ? probs_bytes : opart_bytes);
     L.qf = take(static_cast<uint32_t>(G) * D * 4u);
     L.mail_stride = decode_mail_bytes(row_bytes, br_max_pad);
     L.mail = take(2u * L.mail_stride);
-    L.opart = take(static_cast<uint32_t>(consumer_warps) * G * D * 4u);
+    L.opart = L.probs;
     L.redf = take(2u * kMaxConsumerWarps * 8u * 4u);
     L.red64 = take(kMaxConsumerWarps * 16u);
     L.total = o;
