@@ -230,6 +230,10 @@ def test_prefill_attention_long_prompt(zb):
             ref = torch.nn.functional.scaled_dot_product_attention(
                 Q[:, hq:hq + 1].double(), K[:, hk:hk + 1].double(), V[:, hk:hk + 1].double(), is_causal=True)
             torch.testing.assert_close(out[:, hq:hq + 1].cpu().double(), ref, atol=2e-3, rtol=1e-2)
+            logits = (Q[0, hq].double() @ K[0, hk].double().T) / np.sqrt(float(d))
+            mask = torch.tril(torch.ones(T, T, dtype=torch.bool))
+            ref_lse = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
+            torch.testing.assert_close(lse[0, hq].cpu().double(), ref_lse, atol=1e-4, rtol=1e-5)
     finally:
         cache.close()
 
